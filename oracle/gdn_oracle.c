@@ -1,0 +1,160 @@
+/*
+ * CPU oracle for the gated delta-rule recurrence (TEST INFRASTRUCTURE ONLY).
+ *
+ * This file is the slow, plain definition that the CUDA library is checked
+ * against.  It is used by the tests, by the smoke check and by the benchmark's
+ * CPU-baseline leg; the product path never calls it, and it shares no code,
+ * header, table or helper with the CUDA sources.
+ *
+ * What it computes, per sequence n and value head h (hq = h / (Hv/Hqk)),
+ * independently, in fp64, token by token in order:
+ *
+ *     S <- alpha * S                alpha = exp(g)        (decay first; Section 3.2 "gS")
+ *     a <- S k                      old_v = k^T (gS)      (Section 3.2, old_v)
+ *     d <- beta * (v - a)           delta                 (Section 3.2, delta)
+ *     S <- S + d k^T                S' = gS + k delta^T   (Section 3.2, S')
+ *     o <- S q                      output from the updated state; algebraically
+ *                                   equal to q^T(gS) + delta (q^T k) (Section 3.2)
+ *
+ * which is S_t = alpha_t S_{t-1} (I - beta_t k_t k_t^T) + beta_t v_t k_t^T,
+ * o_t = S_t q_t with the state held as [dv][dk] (the paper writes the transpose).
+ * Inputs are the bf16/fp32 arrays the GPU receives, widened exactly to fp64.
+ * No blocking, fusion or reordering beyond the five lines above.
+ *
+ * Pins (tests/test_oracle_pins.py): one-token closed form, beta = 0 pure decay,
+ * one-hot-key associative recall, the per-step identity for S k, the
+ * orthogonal-key closed form through library matmuls, split/packing invariance,
+ * linearity, V-row independence, brute-force matrix products on tiny inputs, the
+ * paper's K x V form coded separately, and a chunked WY/UT reformulation.
+ */
+#include <math.h>
+#include <pthread.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+static double bf16_to_double(uint16_t b) {
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+typedef struct {
+    const uint16_t *q, *k, *v;
+    const float *g, *beta;
+    const int32_t *cu_seqlens; /* NULL => decode: sequence n is the single token n */
+    const float *initial_state;
+    double *out, *final_state;
+    int num_seqs, Hqk, Hv, dk, dv;
+    int next_unit; /* work counter, guarded by lock */
+    pthread_mutex_t lock;
+} job_t;
+
+/* One (sequence, value-head) unit: the token loop of the definition. */
+static void run_unit(const job_t *J, int n, int h, double *S, double *kk, double *qq) {
+    const int dk = J->dk, dv = J->dv, Hqk = J->Hqk, Hv = J->Hv;
+    const int hq = h / (Hv / Hqk);
+    const int t0 = J->cu_seqlens ? J->cu_seqlens[n] : n;
+    const int t1 = J->cu_seqlens ? J->cu_seqlens[n + 1] : n + 1;
+    const size_t sbase = ((size_t)n * Hv + h) * (size_t)dv * dk;
+
+    for (int r = 0; r < dv; ++r)
+        for (int c = 0; c < dk; ++c)
+            S[(size_t)r * dk + c] = J->initial_state ? (double)J->initial_state[sbase + (size_t)r * dk + c] : 0.0;
+
+    for (int t = t0; t < t1; ++t) {
+        const uint16_t *qt = J->q + ((size_t)t * Hqk + hq) * dk;
+        const uint16_t *kt = J->k + ((size_t)t * Hqk + hq) * dk;
+        const uint16_t *vt = J->v + ((size_t)t * Hv + h) * dv;
+        for (int c = 0; c < dk; ++c) {
+            kk[c] = bf16_to_double(kt[c]);
+            qq[c] = bf16_to_double(qt[c]);
+        }
+        const double alpha = exp((double)J->g[(size_t)t * Hv + h]);
+        const double beta = (double)J->beta[(size_t)t * Hv + h];
+        double *o = J->out + ((size_t)t * Hv + h) * dv;
+        for (int r = 0; r < dv; ++r) {
+            double *Sr = S + (size_t)r * dk;
+            for (int c = 0; c < dk; ++c) Sr[c] *= alpha; /* S <- alpha S   */
+            double a = 0.0;
+            for (int c = 0; c < dk; ++c) a += Sr[c] * kk[c]; /* a = (S k)_r */
+            const double d = beta * (bf16_to_double(vt[r]) - a); /* delta_r   */
+            for (int c = 0; c < dk; ++c) Sr[c] += d * kk[c]; /* S += d k^T  */
+            double acc = 0.0;
+            for (int c = 0; c < dk; ++c) acc += Sr[c] * qq[c]; /* o = S q    */
+            o[r] = acc;
+        }
+    }
+    if (J->final_state)
+        memcpy(J->final_state + sbase, S, sizeof(double) * (size_t)dv * dk);
+}
+
+static void *worker(void *arg) {
+    job_t *J = (job_t *)arg;
+    double *S = (double *)malloc(sizeof(double) * (size_t)J->dv * J->dk);
+    double *kk = (double *)malloc(sizeof(double) * (size_t)J->dk);
+    double *qq = (double *)malloc(sizeof(double) * (size_t)J->dk);
+    const int units = J->num_seqs * J->Hv;
+    for (;;) {
+        pthread_mutex_lock(&J->lock);
+        const int u = J->next_unit++;
+        pthread_mutex_unlock(&J->lock);
+        if (u >= units) break;
+        run_unit(J, u / J->Hv, u % J->Hv, S, kk, qq);
+    }
+    free(S);
+    free(kk);
+    free(qq);
+    return NULL;
+}
+
+static int run_job(job_t *J, int num_threads) {
+    if (J->num_seqs < 0 || J->Hqk <= 0 || J->Hv <= 0 || J->dk <= 0 || J->dv <= 0) return 1;
+    if (J->Hv % J->Hqk != 0) return 1;
+    const int units = J->num_seqs * J->Hv;
+    if (units == 0) return 0;
+    if (num_threads < 1) num_threads = 1;
+    if (num_threads > units) num_threads = units;
+    if (num_threads > 256) num_threads = 256;
+    J->next_unit = 0;
+    pthread_mutex_init(&J->lock, NULL);
+    pthread_t th[256];
+    for (int i = 1; i < num_threads; ++i) pthread_create(&th[i], NULL, worker, J);
+    worker(J);
+    for (int i = 1; i < num_threads; ++i) pthread_join(th[i], NULL);
+    pthread_mutex_destroy(&J->lock);
+    return 0;
+}
+
+/* Varlen prefill.  out: fp64 [T_tot,Hv,dv]; final_state: fp64 [N,Hv,dv,dk] or NULL;
+ * initial_state: fp32 [N,Hv,dv,dk] or NULL (zeros).  Returns 0 on success. */
+int gdn_oracle_prefill(const uint16_t *q, const uint16_t *k, const uint16_t *v, const float *g,
+                       const float *beta, const int32_t *cu_seqlens, const float *initial_state,
+                       double *out, double *final_state, int num_seqs, int Hqk, int Hv, int dk,
+                       int dv, int num_threads) {
+    job_t J;
+    memset(&J, 0, sizeof J);
+    J.q = q; J.k = k; J.v = v; J.g = g; J.beta = beta;
+    J.cu_seqlens = cu_seqlens;
+    J.initial_state = initial_state;
+    J.out = out; J.final_state = final_state;
+    J.num_seqs = num_seqs; J.Hqk = Hqk; J.Hv = Hv; J.dk = dk; J.dv = dv;
+    if (!cu_seqlens) return 1;
+    return run_job(&J, num_threads);
+}
+
+/* Single-token decode: batch item b is a one-token sequence starting from state_in[b]. */
+int gdn_oracle_decode(const uint16_t *q, const uint16_t *k, const uint16_t *v, const float *g,
+                      const float *beta, const float *state_in, double *state_out, double *out,
+                      int B, int Hqk, int Hv, int dk, int dv, int num_threads) {
+    job_t J;
+    memset(&J, 0, sizeof J);
+    J.q = q; J.k = k; J.v = v; J.g = g; J.beta = beta;
+    J.cu_seqlens = NULL;
+    J.initial_state = state_in;
+    J.out = out; J.final_state = state_out;
+    J.num_seqs = B; J.Hqk = Hqk; J.Hv = Hv; J.dk = dk; J.dv = dv;
+    if (!state_in) return 1;
+    return run_job(&J, num_threads);
+}
