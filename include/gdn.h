@@ -1,0 +1,141 @@
+/*
+ * libgdn -- gated delta-rule recurrence of Gated DeltaNet for NVIDIA B200 (sm_100a).
+ *
+ * For every sequence (or batch item) and value head h, with hq = h / (Hv / Hqk):
+ *
+ *     S_t = alpha_t S_{t-1} (I - beta_t k_t k_t^T) + beta_t v_t k_t^T ,   alpha_t = exp(g_t)
+ *     o_t = S_t q_t
+ *
+ * i.e. decay the state, read old_v = S k, form delta = beta (v - old_v), add the
+ * rank-one update delta k^T, and read the output from the updated state (the paper's
+ * Section 3.2 equations, with the state stored transposed: [dv][dk], dk contiguous).
+ *
+ * Conventions shared by every entry point
+ *   - Every data pointer is a DEVICE pointer unless stated otherwise.  The caller owns
+ *     all buffers (destination passing: outputs are pre-allocated by the caller); the
+ *     library allocates no device memory and keeps no reference after it returns.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and return without synchronising.
+ *   - Return value: GDN_OK (0) or a positive gdn_status; on error nothing is enqueued.
+ *     No exceptions, no aborts, no printing.
+ *   - bf16 tensors are passed as `const void*` (2-byte elements); 16-byte alignment is
+ *     required for every tensor pointer.
+ *   - Only dk = dv = 128 is supported; Hv must be a multiple of Hqk (value heads
+ *     h = j*G .. j*G+G-1 share q/k head j, G = Hv/Hqk).
+ *   - The kernels neither normalise q/k nor compute the gates: g is the log-decay
+ *     (alpha = exp(g)) and beta the write strength, both per value head.  There is no
+ *     scale argument: o = S q literally.
+ */
+#ifndef GDN_H_
+#define GDN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum gdn_status {
+    GDN_OK = 0,
+    GDN_ERR_NULL = 1,        /* a required pointer is NULL                                   */
+    GDN_ERR_SHAPE = 2,       /* negative size, Hv % Hqk != 0, max_seqlen inconsistent        */
+    GDN_ERR_UNSUPPORTED = 3, /* dk != 128 or dv != 128, or the device is not sm_100          */
+    GDN_ERR_WORKSPACE = 4,   /* workspace NULL, too small or not 1024-byte aligned           */
+    GDN_ERR_ALIGN = 5,       /* a tensor pointer is not 16-byte aligned                      */
+    GDN_ERR_CUDA = 6         /* the CUDA runtime reported an error while enqueueing          */
+} gdn_status;
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* gdn_status_string(int status);
+
+/*
+ * Single-token decode (Section 3.2: old_v, delta, S' and out, one token per batch item).
+ * Reads each state row once and writes it once in the same pass; the output uses
+ * out = q^T(alpha S) + delta (q^T k), so the updated state is never re-read.
+ *
+ *   q, k      bf16 [B, Hqk, dk]
+ *   v         bf16 [B, Hv, dv]
+ *   g, beta   fp32 [B, Hv]
+ *   state_in  fp32 [B, Hv, dv, dk]
+ *   state_out fp32 [B, Hv, dv, dk]   may be exactly state_in (in place); partial overlap is
+ *                                    undefined
+ *   out       bf16 [B, Hv, dv]       rounded to nearest even from fp32
+ *
+ * B = 0 returns GDN_OK without launching.
+ */
+int gdn_decode(const void* q, const void* k, const void* v, const float* g, const float* beta,
+               const float* state_in, float* state_out, void* out,
+               int B, int Hqk, int Hv, int dk, int dv, void* stream);
+
+/*
+ * gdn_decode with an explicit launch shape (rows per warp x warps per CTA), for tuning
+ * the batch-regime table of Section 5.4 ("decode gap: dispatch and shape split").
+ * variant in [0, gdn_decode_num_variants()); same arguments and result as gdn_decode.
+ */
+int gdn_decode_variant(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                       const float* state_in, float* state_out, void* out,
+                       int B, int Hqk, int Hv, int dk, int dv, int variant, void* stream);
+int gdn_decode_num_variants(void);
+
+/*
+ * Bytes of device scratch that gdn_prefill needs for the given sizes (host-side
+ * arithmetic only; returns 0 for unsupported shapes).  The workspace holds the
+ * per-chunk summaries (the chunk table, the cumulative gates, the UT-transformed
+ * W and T operands and the masked chunk-local attention matrix).
+ */
+size_t gdn_prefill_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv, int dk, int dv);
+
+/*
+ * Variable-length prefill.  The same recurrence as above, evaluated over 64-token
+ * chunks in the chunked WY / UT-transform form (the "chunk-level" reformulation the
+ * paper's Sections 3.3 and 5 point to): inside a chunk the triangular system
+ * (I + strict_lower(diag(beta) (K K^T o D))) is inverted once, the resulting W and U
+ * operands turn the chunk into dense products, and the state is carried serially
+ * from chunk to chunk with those products on the tcgen05 tensor cores.
+ *
+ *   q, k          bf16 [T_tot, Hqk, dk]   sequences packed back to back
+ *   v             bf16 [T_tot, Hv, dv]
+ *   g, beta       fp32 [T_tot, Hv]
+ *   cu_seqlens    int32 [num_seqs+1] on the DEVICE; cu[0] = 0, non-decreasing,
+ *                 cu[num_seqs] = total_tokens.  Zero-length sequences are allowed.
+ *   initial_state fp32 [num_seqs, Hv, dv, dk] or NULL (all zeros)
+ *   out           bf16 [T_tot, Hv, dv]
+ *   final_state   fp32 [num_seqs, Hv, dv, dk] or NULL (not wanted); may alias
+ *                 initial_state exactly
+ *   total_tokens, num_seqs, max_seqlen   host-known sizes (no device sync happens);
+ *                 max_seqlen must be >= the longest sequence and <= total_tokens
+ *   workspace     >= gdn_prefill_workspace_bytes(...) bytes, 1024-byte aligned
+ *
+ * A malformed cu_seqlens can give wrong results but never an out-of-range access:
+ * every token index is clamped to [0, total_tokens).  total_tokens = 0 or
+ * num_seqs = 0 returns GDN_OK without launching.
+ */
+int gdn_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                const int32_t* cu_seqlens, const float* initial_state, void* out, float* final_state,
+                int total_tokens, int num_seqs, int max_seqlen,
+                int Hqk, int Hv, int dk, int dv,
+                void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Token-serial prefill: the same inputs and outputs as gdn_prefill (no workspace),
+ * computed by the per-token recurrence of Section 3.2 with the state rows held in
+ * registers and split along V across thread blocks (the paper's own prefill shape).
+ * Kept for very short sequences and as an on-device cross-check of the chunked path.
+ */
+int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                          const int32_t* cu_seqlens, const float* initial_state, void* out,
+                          float* final_state, int total_tokens, int num_seqs, int max_seqlen,
+                          int Hqk, int Hv, int dk, int dv, void* stream);
+
+/*
+ * Reads (and clears) the device-side status word that the prefill kernels set when a
+ * bounded wait on an asynchronous copy or tensor-core completion ran out.  HOST
+ * pointer out; synchronises `stream`.  *device_status == 0 means no kernel gave up.
+ */
+int gdn_last_device_status(void* workspace, int* device_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GDN_H_ */

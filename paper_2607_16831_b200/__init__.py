@@ -1,0 +1,137 @@
+"""Python binding of libgdn (argument marshalling only; every step runs in the CUDA kernels).
+
+The functions mirror the C entry points of include/gdn.h one to one and take torch CUDA
+tensors (torch is used for device memory and streams only).  There is no CPU fallback:
+if libgdn.so is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libgdn.so")
+
+GDN_OK = 0
+STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL", 2: "GDN_ERR_SHAPE", 3: "GDN_ERR_UNSUPPORTED",
+                4: "GDN_ERR_WORKSPACE", 5: "GDN_ERR_ALIGN", 6: "GDN_ERR_CUDA"}
+
+# Every symbol include/gdn.h declares.
+EXPORTS = ("gdn_status_string", "gdn_decode", "gdn_decode_variant", "gdn_decode_num_variants",
+           "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_recurrent", "gdn_last_device_status")
+
+
+class GdnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s" % (where, status_string(status)))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libgdn.so (built in-tree by paper_2607_16831_b200/build.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("libgdn.so is not built: run `python -m paper_2607_16831_b200.build` "
+                              "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        P, I, Z = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.gdn_status_string.argtypes = [I]
+        L.gdn_status_string.restype = ctypes.c_char_p
+        L.gdn_decode.argtypes = [P] * 8 + [I] * 5 + [P]
+        L.gdn_decode.restype = I
+        L.gdn_decode_variant.argtypes = [P] * 8 + [I] * 6 + [P]
+        L.gdn_decode_variant.restype = I
+        L.gdn_decode_num_variants.argtypes = []
+        L.gdn_decode_num_variants.restype = I
+        L.gdn_prefill_workspace_bytes.argtypes = [I] * 6
+        L.gdn_prefill_workspace_bytes.restype = Z
+        L.gdn_prefill.argtypes = [P] * 9 + [I] * 7 + [P, Z, P]
+        L.gdn_prefill.restype = I
+        L.gdn_prefill_recurrent.argtypes = [P] * 9 + [I] * 7 + [P]
+        L.gdn_prefill_recurrent.restype = I
+        L.gdn_last_device_status.argtypes = [P, ctypes.POINTER(I), P]
+        L.gdn_last_device_status.restype = I
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().gdn_status_string(int(status)).decode()
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else int(t.data_ptr())
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+
+        stream = torch.cuda.current_stream()
+    s = int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
+    return s or None
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != GDN_OK:
+        raise GdnError(rc, where)
+
+
+def gdn_decode(q, k, v, g, beta, state_in, state_out, out, stream=None, variant: int = -1) -> None:
+    """q,k: bf16 [B,Hqk,128]; v,out: bf16 [B,Hv,128]; g,beta: fp32 [B,Hv];
+    state_in/state_out: fp32 [B,Hv,128,128].  Enqueues on `stream` (default: current)."""
+    B, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    args = [_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(state_in), _ptr(state_out), _ptr(out),
+            B, Hqk, Hv, dk, dv]
+    if variant < 0:
+        _check(lib().gdn_decode(*args, _stream(stream)), "gdn_decode")
+    else:
+        _check(lib().gdn_decode_variant(*args, variant, _stream(stream)), "gdn_decode_variant")
+
+
+def gdn_decode_num_variants() -> int:
+    return int(lib().gdn_decode_num_variants())
+
+
+def gdn_prefill_workspace_bytes(total_tokens: int, num_seqs: int, Hqk: int, Hv: int, dk: int = 128,
+                                dv: int = 128) -> int:
+    return int(lib().gdn_prefill_workspace_bytes(total_tokens, num_seqs, Hqk, Hv, dk, dv))
+
+
+def gdn_prefill(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state, max_seqlen: int, workspace,
+                stream=None) -> None:
+    """q,k: bf16 [T,Hqk,128]; v,out: bf16 [T,Hv,128]; g,beta: fp32 [T,Hv]; cu_seqlens: int32 [N+1]
+    (device); initial_state/final_state: fp32 [N,Hv,128,128] or None; workspace: a uint8 CUDA
+    tensor of at least gdn_prefill_workspace_bytes(...) bytes, 1024-byte aligned."""
+    T, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    N = cu_seqlens.shape[0] - 1
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().gdn_prefill(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(cu_seqlens), _ptr(initial_state),
+                           _ptr(out), _ptr(final_state), T, N, int(max_seqlen), Hqk, Hv, dk, dv, _ptr(workspace),
+                           wbytes, _stream(stream))
+    _check(rc, "gdn_prefill")
+
+
+def gdn_prefill_recurrent(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state, max_seqlen: int,
+                          stream=None) -> None:
+    T, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    N = cu_seqlens.shape[0] - 1
+    rc = lib().gdn_prefill_recurrent(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(cu_seqlens),
+                                     _ptr(initial_state), _ptr(out), _ptr(final_state), T, N, int(max_seqlen),
+                                     Hqk, Hv, dk, dv, _stream(stream))
+    _check(rc, "gdn_prefill_recurrent")
+
+
+def gdn_last_device_status(workspace, stream=None) -> int:
+    val = ctypes.c_int(0)
+    _check(lib().gdn_last_device_status(_ptr(workspace), ctypes.byref(val), _stream(stream)),
+           "gdn_last_device_status")
+    return int(val.value)

@@ -1,0 +1,168 @@
+// C-ABI entry points of libgdn: argument validation and launch dispatch only.
+#include "gdn_common.cuh"
+
+namespace gdn {
+cudaError_t decode_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                            const float* s_in, float* s_out, void* out, int B, int Hqk, int Hv, int variant,
+                            cudaStream_t st);
+cudaError_t prefill_recurrent_dispatch(const void* q, const void* k, const void* v, const float* g,
+                                       const float* beta, const int32_t* cu_seqlens, const float* initial_state,
+                                       void* out, float* final_state, int total_tokens, int num_seqs, int Hqk,
+                                       int Hv, cudaStream_t st);
+size_t prefill_chunked_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv);
+cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v, const float* g,
+                                     const float* beta, const int32_t* cu_seqlens, const float* initial_state,
+                                     void* out, float* final_state, int total_tokens, int num_seqs,
+                                     int max_seqlen, int Hqk, int Hv, void* workspace, size_t workspace_bytes,
+                                     cudaStream_t st);
+
+// 1 = sm_100 family, 0 = other, -1 = unknown yet.  Indexed by device ordinal.
+static int g_device_ok[64] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1,
+                              -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1,
+                              -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1,
+                              -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};
+
+static bool device_supported() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (dev < 0 || dev >= 64) return false;
+    if (g_device_ok[dev] < 0) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
+        g_device_ok[dev] = (major == 10) ? 1 : 0;
+    }
+    return g_device_ok[dev] == 1;
+}
+
+static int check_heads(int Hqk, int Hv, int dk, int dv) {
+    if (Hqk <= 0 || Hv <= 0 || dk <= 0 || dv <= 0) return GDN_ERR_SHAPE;
+    if (Hv % Hqk != 0) return GDN_ERR_SHAPE;
+    if (dk != kD || dv != kD) return GDN_ERR_UNSUPPORTED;
+    return GDN_OK;
+}
+
+static int decode_impl(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                       const float* state_in, float* state_out, void* out, int B, int Hqk, int Hv, int dk, int dv,
+                       int variant, void* stream) {
+    if (B < 0) return GDN_ERR_SHAPE;
+    if (int rc = check_heads(Hqk, Hv, dk, dv)) return rc;
+    if (B == 0) return GDN_OK;
+    if (!q || !k || !v || !g || !beta || !state_in || !state_out || !out) return GDN_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
+        !aligned16(state_in) || !aligned16(state_out) || !aligned16(out))
+        return GDN_ERR_ALIGN;
+    if ((long long)B * Hv * 32 > 0x7fffffffLL) return GDN_ERR_SHAPE;
+    if (!device_supported()) return GDN_ERR_UNSUPPORTED;
+    cudaError_t e = decode_dispatch(q, k, v, g, beta, state_in, state_out, out, B, Hqk, Hv, variant,
+                                    (cudaStream_t)stream);
+    return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
+
+static int check_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                         const int32_t* cu_seqlens, const float* initial_state, void* out, float* final_state,
+                         int total_tokens, int num_seqs, int max_seqlen, int Hqk, int Hv, int dk, int dv,
+                         bool* nothing_to_do) {
+    *nothing_to_do = false;
+    if (total_tokens < 0 || num_seqs < 0 || max_seqlen < 0) return GDN_ERR_SHAPE;
+    if (int rc = check_heads(Hqk, Hv, dk, dv)) return rc;
+    if (max_seqlen > total_tokens) return GDN_ERR_SHAPE;
+    if (total_tokens > 0 && (num_seqs == 0 || max_seqlen == 0)) return GDN_ERR_SHAPE;
+    if ((long long)max_seqlen * num_seqs < total_tokens) return GDN_ERR_SHAPE;
+    if (num_seqs == 0) { *nothing_to_do = true; return GDN_OK; }
+    if (!cu_seqlens) return GDN_ERR_NULL;
+    if (total_tokens > 0 && (!q || !k || !v || !g || !beta || !out)) return GDN_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
+        !aligned16(out) || !aligned16(initial_state) || !aligned16(final_state) ||
+        (reinterpret_cast<uintptr_t>(cu_seqlens) & 3u))
+        return GDN_ERR_ALIGN;
+    if ((long long)num_seqs * Hv * 16 > 0x7fffffffLL) return GDN_ERR_SHAPE;
+    if (!device_supported()) return GDN_ERR_UNSUPPORTED;
+    return GDN_OK;
+}
+
+}  // namespace gdn
+
+using namespace gdn;
+
+extern "C" {
+
+const char* gdn_status_string(int status) {
+    switch (status) {
+        case GDN_OK: return "GDN_OK";
+        case GDN_ERR_NULL: return "GDN_ERR_NULL: a required pointer is NULL";
+        case GDN_ERR_SHAPE: return "GDN_ERR_SHAPE: inconsistent or negative sizes";
+        case GDN_ERR_UNSUPPORTED: return "GDN_ERR_UNSUPPORTED: head size other than 128 or device is not sm_100";
+        case GDN_ERR_WORKSPACE: return "GDN_ERR_WORKSPACE: workspace missing, too small or misaligned";
+        case GDN_ERR_ALIGN: return "GDN_ERR_ALIGN: a tensor pointer is not 16-byte aligned";
+        case GDN_ERR_CUDA: return "GDN_ERR_CUDA: the CUDA runtime reported an error";
+        default: return "GDN_ERR_UNKNOWN";
+    }
+}
+
+int gdn_decode(const void* q, const void* k, const void* v, const float* g, const float* beta,
+               const float* state_in, float* state_out, void* out, int B, int Hqk, int Hv, int dk, int dv,
+               void* stream) {
+    return decode_impl(q, k, v, g, beta, state_in, state_out, out, B, Hqk, Hv, dk, dv, -1, stream);
+}
+
+int gdn_decode_variant(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                       const float* state_in, float* state_out, void* out, int B, int Hqk, int Hv, int dk, int dv,
+                       int variant, void* stream) {
+    if (variant < 0 || variant >= gdn_decode_num_variants()) return GDN_ERR_SHAPE;
+    return decode_impl(q, k, v, g, beta, state_in, state_out, out, B, Hqk, Hv, dk, dv, variant, stream);
+}
+
+int gdn_decode_num_variants(void) { return 10; }
+
+size_t gdn_prefill_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv, int dk, int dv) {
+    if (total_tokens < 0 || num_seqs < 0) return 0;
+    if (check_heads(Hqk, Hv, dk, dv) != GDN_OK) return 0;
+    return prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv);
+}
+
+int gdn_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                const int32_t* cu_seqlens, const float* initial_state, void* out, float* final_state,
+                int total_tokens, int num_seqs, int max_seqlen, int Hqk, int Hv, int dk, int dv,
+                void* workspace, size_t workspace_bytes, void* stream) {
+    bool nothing = false;
+    if (int rc = check_prefill(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state, total_tokens,
+                               num_seqs, max_seqlen, Hqk, Hv, dk, dv, &nothing))
+        return rc;
+    if (nothing) return GDN_OK;
+    const size_t need = prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv);
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
+        return GDN_ERR_WORKSPACE;
+    cudaError_t e = prefill_chunked_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
+                                             total_tokens, num_seqs, max_seqlen, Hqk, Hv, workspace,
+                                             workspace_bytes, (cudaStream_t)stream);
+    return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
+
+int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                          const int32_t* cu_seqlens, const float* initial_state, void* out, float* final_state,
+                          int total_tokens, int num_seqs, int max_seqlen, int Hqk, int Hv, int dk, int dv,
+                          void* stream) {
+    bool nothing = false;
+    if (int rc = check_prefill(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state, total_tokens,
+                               num_seqs, max_seqlen, Hqk, Hv, dk, dv, &nothing))
+        return rc;
+    if (nothing) return GDN_OK;
+    cudaError_t e = prefill_recurrent_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
+                                               total_tokens, num_seqs, Hqk, Hv, (cudaStream_t)stream);
+    return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
+
+int gdn_last_device_status(void* workspace, int* device_status, void* stream) {
+    if (!workspace || !device_status) return GDN_ERR_NULL;
+    int val = 0;
+    if (cudaMemcpyAsync(&val, workspace, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+        return GDN_ERR_CUDA;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return GDN_ERR_CUDA;
+    *device_status = val;
+    if (val != 0) {
+        if (cudaMemsetAsync(workspace, 0, sizeof(int), (cudaStream_t)stream) != cudaSuccess) return GDN_ERR_CUDA;
+    }
+    return GDN_OK;
+}
+
+}  // extern "C"

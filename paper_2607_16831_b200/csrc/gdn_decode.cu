@@ -1,0 +1,152 @@
+// Single-token decode of the gated delta rule (Section 3.2 of the paper):
+//     old_v = k^T (alpha S),  delta = beta (v - old_v),  S' = alpha S + delta k^T,
+//     out   = q^T (alpha S) + delta (q^T k)
+// One pass over the fp32 state: every row is read once, updated in registers and
+// written once; the output comes from the decayed old row plus a scalar correction,
+// so the new state is never re-read.
+//
+// Work split.  A state row is 128 fp32 = 512 B.  Eight lanes own one row (each lane
+// holds four float4 of it, interleaved so that every load instruction of a warp
+// covers four whole 128-byte segments), so a warp works on four rows per "batch" and
+// both dot products of a row reduce with three shuffle steps inside the 8-lane group.
+// A warp issues the loads of all of its NB batches before the first use, which keeps
+// NB*64 bytes per lane in flight; the V dimension is split over warps and CTAs so
+// that small batches still cover all SMs.
+#include "gdn_common.cuh"
+
+namespace gdn {
+
+template <int NB>
+__device__ __forceinline__ void decode_rows(const float* __restrict__ s_in, float* __restrict__ s_out,
+                                            const uint16_t* __restrict__ v_h, uint16_t* __restrict__ o_h,
+                                            int row0, const float (&kf)[16], const float (&qf)[16],
+                                            float alpha, float beta, float qk, int sub, int c) {
+    float4 s[NB][4];
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
+        const float4* src = reinterpret_cast<const float4*>(s_in + (size_t)(row0 + i * 4 + sub) * kD);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) s[i][j] = __ldcs(src + c + 8 * j);
+    }
+    float vr[NB];
+#pragma unroll
+    for (int i = 0; i < NB; ++i) vr[i] = bf16_bits_to_float(v_h[row0 + i * 4 + sub]);
+
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
+        float a = 0.f, p = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            a = fmaf(s[i][j].x, kf[4 * j + 0], a);
+            a = fmaf(s[i][j].y, kf[4 * j + 1], a);
+            a = fmaf(s[i][j].z, kf[4 * j + 2], a);
+            a = fmaf(s[i][j].w, kf[4 * j + 3], a);
+            p = fmaf(s[i][j].x, qf[4 * j + 0], p);
+            p = fmaf(s[i][j].y, qf[4 * j + 1], p);
+            p = fmaf(s[i][j].z, qf[4 * j + 2], p);
+            p = fmaf(s[i][j].w, qf[4 * j + 3], p);
+        }
+#pragma unroll
+        for (int m = 1; m < 8; m <<= 1) {
+            a += __shfl_xor_sync(0xffffffffu, a, m);
+            p += __shfl_xor_sync(0xffffffffu, p, m);
+        }
+        const float delta = beta * (vr[i] - alpha * a);
+        float4* dst = reinterpret_cast<float4*>(s_out + (size_t)(row0 + i * 4 + sub) * kD);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float4 w;
+            w.x = fmaf(alpha, s[i][j].x, delta * kf[4 * j + 0]);
+            w.y = fmaf(alpha, s[i][j].y, delta * kf[4 * j + 1]);
+            w.z = fmaf(alpha, s[i][j].z, delta * kf[4 * j + 2]);
+            w.w = fmaf(alpha, s[i][j].w, delta * kf[4 * j + 3]);
+            __stcs(dst + c + 8 * j, w);
+        }
+        if (c == 0) o_h[row0 + i * 4 + sub] = float_to_bf16_bits(fmaf(delta, qk, alpha * p));
+    }
+}
+
+// grid.x = B*Hv*SPLIT, block = WARPS*32.  Each CTA owns 128/SPLIT rows of one head and
+// each warp 4*NB of them: 128 = SPLIT * WARPS * 4 * NB.
+template <int NB, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32)
+gdn_decode_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
+                  const uint16_t* __restrict__ v, const float* __restrict__ g,
+                  const float* __restrict__ beta, const float* s_in, float* s_out,
+                  uint16_t* __restrict__ out, int Hqk, int Hv, int split) {
+    const int cta = blockIdx.x;
+    const int part = cta % split;
+    const int bh = cta / split;  // b*Hv + h
+    const int h = bh % Hv;
+    const int b = bh / Hv;
+    const int hq = h / (Hv / Hqk);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane >> 3, c = lane & 7;
+    const int row0 = (part * WARPS + warp) * (4 * NB);
+
+    // q, k columns of this lane: float4 index c + 8j  <->  bf16 elements 4(c+8j) .. +3
+    const uint2* k4 = reinterpret_cast<const uint2*>(k + ((size_t)b * Hqk + hq) * kD);
+    const uint2* q4 = reinterpret_cast<const uint2*>(q + ((size_t)b * Hqk + hq) * kD);
+    float kf[16], qf[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint2 kw = __ldg(k4 + c + 8 * j);
+        const uint2 qw = __ldg(q4 + c + 8 * j);
+        unpack_bf16x2(kw.x, kf[4 * j + 0], kf[4 * j + 1]);
+        unpack_bf16x2(kw.y, kf[4 * j + 2], kf[4 * j + 3]);
+        unpack_bf16x2(qw.x, qf[4 * j + 0], qf[4 * j + 1]);
+        unpack_bf16x2(qw.y, qf[4 * j + 2], qf[4 * j + 3]);
+    }
+    const float alpha = __expf(__ldg(g + bh));
+    const float bt = __ldg(beta + bh);
+    float qk = 0.f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) qk = fmaf(qf[j], kf[j], qk);
+#pragma unroll
+    for (int m = 1; m < 8; m <<= 1) qk += __shfl_xor_sync(0xffffffffu, qk, m);
+
+    const size_t sbase = (size_t)bh * kD * kD;
+    decode_rows<NB>(s_in + sbase, s_out + sbase, v + (size_t)bh * kD, out + (size_t)bh * kD, row0, kf, qf,
+                    alpha, bt, qk, sub, c);
+}
+
+template <int NB, int WARPS>
+static cudaError_t launch(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                          const float* s_in, float* s_out, void* out, int B, int Hqk, int Hv,
+                          cudaStream_t st) {
+    constexpr int split = kD / (WARPS * 4 * NB);
+    static_assert(split >= 1 && split * WARPS * 4 * NB == kD, "rows must tile the head");
+    const long long ctas = (long long)B * Hv * split;
+    gdn_decode_kernel<NB, WARPS><<<(unsigned)ctas, WARPS * 32, 0, st>>>(
+        (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta, s_in, s_out, (uint16_t*)out,
+        Hqk, Hv, split);
+    return cudaGetLastError();
+}
+
+// Launch-shape table.  `variant` < 0 picks from the batch size: below ~16 items the
+// kernel is latency bound and wants as many small CTAs as possible (one warp, four
+// rows: 1024 CTAs at B = 1); large batches want more bytes in flight per warp.
+cudaError_t decode_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                            const float* s_in, float* s_out, void* out, int B, int Hqk, int Hv,
+                            int variant, cudaStream_t st) {
+    if (variant < 0) {
+        if (B <= 2) variant = 0;
+        else if (B <= 16) variant = 1;
+        else variant = 3;
+    }
+    switch (variant) {
+        case 0: return launch<1, 1>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
+        case 1: return launch<2, 1>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
+        case 2: return launch<2, 2>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
+        case 3: return launch<2, 4>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
+        case 4: return launch<4, 2>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
+        case 5: return launch<4, 4>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
+        case 6: return launch<4, 8>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
+        case 7: return launch<8, 4>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
+        case 8: return launch<1, 4>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
+        case 9: return launch<2, 8>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace gdn

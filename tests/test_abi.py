@@ -1,0 +1,72 @@
+"""The C-ABI library: loads without a GPU, exports every symbol the header declares, and
+rejects bad arguments on the host before touching a device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def gdn():
+    from paper_2607_16831_b200 import build
+    build.build()
+    import paper_2607_16831_b200 as g
+    return g
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "gdn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gdn_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_and_binding_agree(gdn):
+    names = declared_functions()
+    assert sorted(gdn.EXPORTS) == names
+    L = gdn.lib()
+    for n in names:
+        assert getattr(L, n) is not None
+
+
+def test_status_strings(gdn):
+    assert gdn.status_string(0) == "GDN_OK"
+    for code, name in gdn.STATUS_NAMES.items():
+        assert gdn.status_string(code).startswith(name)
+    assert "UNKNOWN" in gdn.status_string(99)
+
+
+def test_host_side_argument_checks(gdn):
+    L = gdn.lib()
+    fake = ctypes.c_void_p(0x1000)  # never dereferenced: every call below fails validation first
+    odd = ctypes.c_void_p(0x1004)
+    # decode
+    assert L.gdn_decode(None, None, None, None, None, None, None, None, 0, 16, 32, 128, 128, None) == 0
+    assert L.gdn_decode(None, fake, fake, fake, fake, fake, fake, fake, 2, 16, 32, 128, 128, None) == 1
+    assert L.gdn_decode(fake, fake, fake, fake, fake, fake, fake, fake, -1, 16, 32, 128, 128, None) == 2
+    assert L.gdn_decode(fake, fake, fake, fake, fake, fake, fake, fake, 2, 16, 33, 128, 128, None) == 2
+    assert L.gdn_decode(fake, fake, fake, fake, fake, fake, fake, fake, 2, 16, 32, 64, 128, None) == 3
+    assert L.gdn_decode(fake, fake, fake, fake, fake, odd, fake, fake, 2, 16, 32, 128, 128, None) == 5
+    assert L.gdn_decode_variant(fake, fake, fake, fake, fake, fake, fake, fake, 2, 16, 32, 128, 128, 99, None) == 2
+    # prefill
+    assert L.gdn_prefill_workspace_bytes(4096, 1, 16, 32, 128, 128) > 0
+    assert L.gdn_prefill_workspace_bytes(4096, 1, 16, 32, 64, 128) == 0
+    args = [fake] * 9
+    assert L.gdn_prefill(*args, 0, 0, 0, 16, 32, 128, 128, None, 0, None) == 0
+    assert L.gdn_prefill(*args, 100, 2, 101, 16, 32, 128, 128, fake, 1 << 30, None) == 2  # max_seqlen > total
+    assert L.gdn_prefill(*args, 100, 2, 10, 16, 32, 128, 128, fake, 1 << 30, None) == 2   # 2*10 < 100
+    assert L.gdn_prefill(*args, 100, 0, 0, 16, 32, 128, 128, fake, 1 << 30, None) == 2
+    a = list(args); a[5] = None
+    assert L.gdn_prefill(*a, 100, 2, 60, 16, 32, 128, 128, fake, 1 << 30, None) == 1     # cu_seqlens NULL
+    a = list(args); a[0] = odd
+    assert L.gdn_prefill(*a, 100, 2, 60, 16, 32, 128, 128, fake, 1 << 30, None) == 5
+    assert L.gdn_prefill_recurrent(*args, 100, 2, 101, 16, 32, 128, 128, None) == 2
+
+
+def test_workspace_size_grows_with_tokens(gdn):
+    a = gdn.gdn_prefill_workspace_bytes(64, 1, 1, 1)
+    b = gdn.gdn_prefill_workspace_bytes(4096, 1, 16, 32)
+    c = gdn.gdn_prefill_workspace_bytes(4096, 16, 16, 32)
+    assert 0 < a < b <= c
