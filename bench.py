@@ -1,0 +1,438 @@
+#!/usr/bin/env python
+"""Benchmark of libgdn on B200.
+
+Default line (N = 1): the decode workload at batch 64 (16 q/k heads, 32 value heads,
+d = 128, fp32 state [64,32,128,128] updated into a separate buffer).  A step is one
+gdn_decode call = one pass over the state.  `value` is state bytes moved per second
+(read + write, 4,194,304 B per batch item) with every buffer resident in HBM; the state
+buffers rotate over > 512 MB so that no step finds its state in L2.  The same JSON line
+carries the prefill workloads (tokens/s with both roofline fractions), the decode batch
+sweep, the roofline of the dominant kernel, and the CPU oracle timed on this machine.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--quick]
+
+With N > 1 (launched by torchrun) every rank runs its own batch of 64 (independent
+shards, no collective on the data path); times are the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+STATE_BYTES_PER_ITEM = 2 * 32 * 128 * 128 * 4           # read + write of one batch item's state
+TOKEN_BYTES_PER_ITEM = 2 * 16 * 128 * 2 + 2 * 32 * 128 * 2 + 2 * 32 * 4   # q,k + v,out + g,beta
+PREFILL_BYTES_PER_TOKEN = 24832                          # q 4096 + k 4096 + v 8192 + out 8192 + g,beta 256
+PREFILL_FLOPS_PER_TOKEN = 5.77e6                         # 11.53 MFLOP per (chunk, value head) / 64 * 32
+# DRAM bytes per decode launch at B = 64 from the committed ncu capture
+# (profiles/decode_b64_ncu.md); None until a capture exists.
+DECODE_B64_DRAM_TRAFFIC = None
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=float(d["hbm_gbs"]), bf16=float(d["bf16_tflops"]),
+                    bf16_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+            nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": (float(np.median(self.samples)) if self.samples else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_device_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ---------------------------------------------------------------------------------- reference arm
+def run_reference(args):
+    """Times the fp64 CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    from gdn_inputs import config
+
+    cfg = config("decode_b64", B=64)
+    tok = cfg["tokens"]
+    cores = oracle.default_threads()
+    for _ in range(args.warmup):
+        oracle.decode(tok.q, tok.k, tok.v, tok.g, tok.beta, cfg["state"])
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.decode(tok.q, tok.k, tok.v, tok.g, tok.beta, cfg["state"])
+    dt = (time.perf_counter() - t0) / max(1, args.steps)
+    val = 64 * STATE_BYTES_PER_ITEM / dt / 1e9
+    line = {
+        "impl": "reference", "metric": "gdn_decode_state_hbm_gbps", "value": val, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "decode_b64", "B": 64, "Hqk": 16, "Hv": 32, "d": 128},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                         "sample": "the full batch-64 decode workload per step"},
+        "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------- GPU arm
+def time_graph(fn_enqueue, iters, reps=5):
+    """Device time per call of `iters` back-to-back calls captured in one CUDA graph."""
+    import torch
+
+    st = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        with torch.cuda.graph(g, stream=st):
+            for i in range(iters):
+                fn_enqueue(i)
+    torch.cuda.synchronize()
+    g.replay()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b) * 1e3 / iters)
+    return float(np.median(ts)), float(np.min(ts))
+
+
+def decode_buffers(B, seed=0, min_footprint=600e6):
+    import torch
+    from gdn_inputs import config
+    from paper_2607_16831_b200 import harness
+
+    cfg = config("decode_b64", B=B, seed=seed)
+    d = harness.to_device(cfg["tokens"])
+    per = B * 32 * 128 * 128 * 4
+    nbuf = max(2, min(64, int(min_footprint // (2 * per)) + 1))
+    base = torch.from_numpy(cfg["state"]).cuda()
+    s_in = [base.clone() for _ in range(nbuf)]
+    s_out = [torch.empty_like(base) for _ in range(nbuf)]
+    out = torch.empty((B, 32, 128), dtype=torch.bfloat16, device="cuda")
+    return cfg, d, s_in, s_out, out, nbuf
+
+
+def bench_prefill(name, peaks, reps, **over):
+    """Whole-call device time of gdn_prefill (prep + intra-chunk + chain kernels)."""
+    import torch
+    import paper_2607_16831_b200 as gdn
+    from gdn_inputs import config
+    from paper_2607_16831_b200 import harness
+
+    cfg = config(name, **over)
+    tok = cfg["tokens"]
+    d = harness.to_device(tok)
+    cu_np = np.asarray(cfg["cu_seqlens"], dtype=np.int32)
+    cu = torch.from_numpy(cu_np).cuda()
+    N = len(cu_np) - 1
+    max_len = int(np.max(np.diff(cu_np)))
+    init = None if cfg["initial_state"] is None else torch.from_numpy(cfg["initial_state"]).cuda()
+    out = torch.empty((tok.T, tok.Hv, 128), dtype=torch.bfloat16, device="cuda")
+    fin = torch.empty((N, tok.Hv, 128, 128), dtype=torch.float32, device="cuda")
+    ws = harness.alloc_workspace(tok.T, N, tok.Hqk, tok.Hv)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")
+
+    def call():
+        gdn.gdn_prefill(d["q"], d["k"], d["v"], d["g"], d["beta"], cu, init, out, fin, max_len, ws)
+
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    assert gdn.gdn_last_device_status(ws) == 0
+    ts = []
+    for _ in range(reps):
+        flush.fill_(1)  # evict L2 (126 MB) between timed calls
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(200000)  # let the launches queue up behind a short spin
+        a.record()
+        call()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b) * 1e-3)
+    t = float(np.median(ts))
+    nstate = (1 if init is not None else 0) + 1
+    alg_bytes = tok.T * PREFILL_BYTES_PER_TOKEN * (tok.Hv / 32.0) + nstate * N * tok.Hv * 65536
+    flops = tok.T * PREFILL_FLOPS_PER_TOKEN * (tok.Hv / 32.0)
+    return {
+        "workload": name, "tokens": int(tok.T), "num_seqs": int(N), "us": t * 1e6, "tokens_per_s": tok.T / t,
+        "hbm": {"achieved_gbs": alg_bytes / t / 1e9, "frac": alg_bytes / t / 1e9 / peaks["hbm"]},
+        "tensor": {"achieved_tflops": flops / t / 1e12, "frac": flops / t / 1e12 / peaks["bf16"]},
+        "chain_steps": int(np.max((np.diff(cu_np) + 63) // 64)),
+        "l2": "256 MB written between timed calls",
+    }
+
+
+def run_gpu(args):
+    import torch
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+
+        dist = dist_
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    import paper_2607_16831_b200 as gdn
+    from paper_2607_16831_b200 import harness
+    from paper_2607_16831_b200.sharding import shard_range
+
+    peaks = load_peaks()
+    B = 64
+    # Every rank owns one whole batch of 64 (weak scaling); shard_range is the same helper
+    # a caller would use to split one global batch across ranks.
+    lo, hi = shard_range(B * world, world, rank)
+    assert hi - lo == B
+    cfg, d, s_in, s_out, out, nbuf = decode_buffers(B, seed=rank)
+
+    def call(i):
+        gdn.gdn_decode(d["q"], d["k"], d["v"], d["g"], d["beta"], s_in[i % nbuf], s_out[i % nbuf], out)
+
+    for i in range(max(3, args.warmup)):
+        call(i)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(physical_device_index(local_rank)) as clk:
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(2000000)  # ~1 ms spin so the host runs ahead of the device
+        a.record()
+        for i in range(args.steps):
+            call(i)
+        b.record()
+        torch.cuda.synchronize()
+    elapsed_ms = a.elapsed_time(b)
+    if dist is not None:
+        t = torch.tensor([elapsed_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+        dist.barrier()
+    ms_per_step = elapsed_ms / args.steps
+    value = world * B * STATE_BYTES_PER_ITEM / (ms_per_step * 1e-3) / 1e9
+
+    line = None
+    if rank == 0:
+        alg_bytes = B * (STATE_BYTES_PER_ITEM + TOKEN_BYTES_PER_ITEM)
+        achieved = alg_bytes / (ms_per_step * 1e-3) / 1e9
+        line = {
+            "metric": "gdn_decode_state_hbm_gbps", "value": value, "unit": "GB/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step,
+            "us_per_call": ms_per_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "decode_b64", "B_per_gpu": B, "Hqk": 16, "Hv": 32, "d": 128,
+                       "state": "fp32 [64,32,128,128] into a separate buffer",
+                       "l2": "state buffers rotate over %d distinct in/out pairs (%.0f MB) so inputs exceed the 126 MB L2"
+                             % (nbuf, 2 * nbuf * B * 32 * 128 * 128 * 4 / 1e6)},
+            "clocks": clk.summary(),
+            "gpu_launches": args.steps,
+            "roofline": {"bound": "hbm", "kernel": "gdn_decode_kernel", "achieved": achieved, "peak": peaks["hbm"],
+                         "unit": "GB/s", "frac": achieved / peaks["hbm"], "peak_source": "of " + peaks["source"],
+                         "frac_of_8TBs_datasheet": achieved / 8000.0, "traffic": DECODE_B64_DRAM_TRAFFIC,
+                         "algorithmic_bytes_per_launch": alg_bytes},
+            "paper_context": {"decode_us": 9.315, "prefill_us": 239.48,
+                              "note": "other workload mix (4/8 heads, contest shapes); context only"},
+        }
+
+    # ---- end-to-end: host buffers, H2D of every input and D2H of every result inside the timed region
+    if rank == 0 or dist is not None:
+        tok = cfg["tokens"]
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+        h_in = [pin(tok.q.view(np.int16)), pin(tok.k.view(np.int16)), pin(tok.v.view(np.int16)), pin(tok.g),
+                pin(tok.beta)]
+        h_state = pin(cfg["state"])
+        h_out = torch.empty((B, 32, 128), dtype=torch.int16).pin_memory()
+        h_state_out = torch.empty_like(h_state).pin_memory()
+        d_in = [torch.empty_like(x, device="cuda") for x in h_in]
+        d_state, d_state_out = s_in[0], s_out[0]
+        d_out16 = out.view(torch.int16)
+
+        def e2e_step(with_state):
+            for hsrc, ddst in zip(h_in, d_in):
+                ddst.copy_(hsrc, non_blocking=True)
+            if with_state:
+                d_state.copy_(h_state, non_blocking=True)
+            gdn.gdn_decode(d_in[0].view(torch.bfloat16), d_in[1].view(torch.bfloat16), d_in[2].view(torch.bfloat16),
+                           d_in[3], d_in[4], d_state, d_state_out, out)
+            h_out.copy_(d_out16, non_blocking=True)
+            if with_state:
+                h_state_out.copy_(d_state_out, non_blocking=True)
+
+        def e2e_time(with_state, steps):
+            for _ in range(3):
+                e2e_step(with_state)
+            torch.cuda.synchronize()
+            if dist is not None:
+                dist.barrier()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(steps):
+                e2e_step(with_state)
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b)
+            if dist is not None:
+                t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                ms = float(t.item())
+            return ms / steps
+
+        tok_in = sum(x.numel() * x.element_size() for x in h_in)
+        ms_full = e2e_time(True, 20)
+        ms_res = e2e_time(False, 200)
+        if rank == 0:
+            line["e2e"] = {"value": world * B * STATE_BYTES_PER_ITEM / (ms_full * 1e-3) / 1e9, "unit": "GB/s",
+                           "ms_per_step": ms_full,
+                           "h2d_bytes_per_step": tok_in + h_state.numel() * 4,
+                           "d2h_bytes_per_step": h_out.numel() * 2 + h_state.numel() * 4,
+                           "note": "every input (tokens and the 134 MB state) copied from pinned host memory and "
+                                   "every result copied back each step; PCIe-bound by construction"}
+            line["e2e_state_resident"] = {"value": world * B * STATE_BYTES_PER_ITEM / (ms_res * 1e-3) / 1e9,
+                                          "unit": "GB/s", "ms_per_step": ms_res, "h2d_bytes_per_step": tok_in,
+                                          "d2h_bytes_per_step": h_out.numel() * 2,
+                                          "note": "the recurrent state stays on the device between steps (the "
+                                                  "serving case); tokens in and outputs back over PCIe each step"}
+
+    if rank == 0 and world == 1:
+        # ---- decode batch sweep: pure device time per call from a CUDA graph of back-to-back calls
+        sweep = []
+        for Bs in ([8, 64] if args.quick else [1, 8, 32, 64, 128, 256]):
+            cfg_s, ds, si, so, oo, nb = decode_buffers(Bs)
+            med, mn = time_graph(lambda i: gdn.gdn_decode(ds["q"], ds["k"], ds["v"], ds["g"], ds["beta"], si[i % nb],
+                                                          so[i % nb], oo), iters=40)
+            gbs = Bs * STATE_BYTES_PER_ITEM / med / 1e3
+            sweep.append({"B": Bs, "us_per_call": med, "us_min": mn, "state_gbs": gbs, "frac_measured": gbs / peaks["hbm"],
+                          "frac_8TBs": gbs / 8000.0, "regime": "latency-bound" if Bs < 8 else "bandwidth-bound"})
+            del cfg_s, ds, si, so, oo
+            torch.cuda.empty_cache()
+        line["decode_sweep"] = {"timing": "40 back-to-back calls in one CUDA graph, cold (rotating) state buffers",
+                                "points": sweep}
+        # ---- prefill workloads
+        pre = []
+        reps = 5 if args.quick else 15
+        pre.append(dict(bench_prefill("prefill_long", peaks, reps), variant="zero initial state"))
+        pre.append(dict(bench_prefill("prefill_long", peaks, reps, initial=True), variant="N(0,0.02) initial state"))
+        pre.append(dict(bench_prefill("prefill_varlen", peaks, reps), variant="16 sequences U[1,2048]"))
+        line["prefill"] = {"rooflines": {"hbm_gbs": peaks["hbm"], "bf16_tflops": peaks["bf16"], "source": peaks["source"],
+                                         "bytes_per_token": PREFILL_BYTES_PER_TOKEN,
+                                         "flops_per_token": PREFILL_FLOPS_PER_TOKEN}, "runs": pre}
+        # ---- CPU oracle on this machine's host cores (reported baseline, not the target)
+        import oracle
+
+        tokc = cfg["tokens"]
+        oracle.decode(tokc.q, tokc.k, tokc.v, tokc.g, tokc.beta, cfg["state"])
+        ts = []
+        for _ in range(3):
+            t0 = time.perf_counter()
+            oracle.decode(tokc.q, tokc.k, tokc.v, tokc.g, tokc.beta, cfg["state"])
+            ts.append(time.perf_counter() - t0)
+        line["cpu_baseline"] = {"value": B * STATE_BYTES_PER_ITEM / min(ts) / 1e9, "unit": "GB/s",
+                                "us_per_call": min(ts) * 1e6, "cores": oracle.default_threads(), "kind": "oracle",
+                                "sample": "the full batch-64 decode workload, best of 3"}
+        if not args.quick:
+            from gdn_inputs import config as mkcfg
+
+            pc = mkcfg("prefill_long", T=1024)
+            pt = pc["tokens"]
+            t0 = time.perf_counter()
+            oracle.prefill(pt.q, pt.k, pt.v, pt.g, pt.beta, pc["cu_seqlens"], None)
+            dt = time.perf_counter() - t0
+            line["cpu_baseline"]["prefill"] = {"tokens_per_s": 1024 / dt, "sample": "first 1024 tokens of the T=4096 "
+                                               "workload (32 value heads), one run", "seconds": dt}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="gdn", choices=["gdn", "reference"])
+    ap.add_argument("--quick", action="store_true", help="shorter sweep and fewer prefill repetitions")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 5 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args)
+    else:
+        args.steps = 2000 if args.steps is None else args.steps
+        args.warmup = 20 if args.warmup is None else args.warmup
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

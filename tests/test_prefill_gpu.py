@@ -1,0 +1,95 @@
+"""Chunked (tcgen05/TMA) prefill parity against the fp64 CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+
+import oracle
+from gdn_inputs import config, make_cu_seqlens, make_state, make_tokens
+from paper_2607_16831_b200 import harness
+
+pytestmark = pytest.mark.gpu
+
+
+def check(cfg, what, **kw):
+    res = harness.run_prefill(cfg, **kw)
+    assert res["device_status"] == 0, "%s: a bounded device wait ran out" % what
+    ref_o, ref_s = oracle.prefill(*harness.token_arrays(cfg["tokens"]), cfg["cu_seqlens"], cfg["initial_state"])
+    e = harness.assert_close(res["out"], ref_o, res["final_state"], ref_s, what)
+    print(what, e)
+    return e
+
+
+def custom(lengths, Hqk, Hv, seed, initial=True, **tok_kw):
+    T = int(np.sum(lengths))
+    tok = make_tokens(T, Hqk, Hv, seed=seed, **tok_kw)
+    init = make_state(len(lengths), Hv, seed=seed) if initial else None
+    return dict(kind="prefill", tokens=tok, cu_seqlens=make_cu_seqlens(lengths), initial_state=init, N=len(lengths))
+
+
+def test_prefill_tiny_config():
+    check(config("prefill_tiny"), "prefill tiny (1 x 64, 1 head)")
+
+
+@pytest.mark.parametrize("T", [1, 63, 64, 65, 130])
+def test_prefill_single_sequence_lengths(T):
+    check(custom([T], 1, 2, seed=T), "prefill T=%d" % T)
+
+
+def test_prefill_two_chunks_no_initial_state():
+    check(custom([128], 2, 4, seed=5, initial=False), "prefill 128 zero-init")
+
+
+def test_prefill_varlen_small_with_empty_sequence():
+    cfg = custom([70, 0, 1, 200, 64], 2, 4, seed=7)
+    res = harness.run_prefill(cfg)
+    np.testing.assert_array_equal(res["final_state"][1], cfg["initial_state"][1].astype(np.float64))
+    check(cfg, "prefill varlen small")
+
+
+def test_prefill_weak_decay_carries_state_across_chunks():
+    # mean log-gate ~ -0.0025: the initial state is still visible after 8 chunks
+    e = check(custom([512], 2, 4, seed=11, gate_mean=6.0), "prefill weak decay")
+    assert e["state_rel_fro"] < 2.5e-3
+
+
+def test_prefill_matches_token_serial_kernel():
+    cfg = custom([300, 77], 2, 4, seed=13)
+    a = harness.run_prefill(cfg)
+    b = harness.run_prefill(cfg, recurrent=True)
+    assert harness.rel_fro(a["out"], b["out"]) < 8e-3
+    assert harness.rel_fro(a["final_state"], b["final_state"]) < 5e-3
+
+
+def test_prefill_final_state_not_requested():
+    cfg = custom([100], 1, 1, seed=17)
+    res = harness.run_prefill(cfg, want_final=False)
+    ref_o, _ = oracle.prefill(*harness.token_arrays(cfg["tokens"]), cfg["cu_seqlens"], cfg["initial_state"])
+    harness.assert_close(res["out"], ref_o, None, None, "prefill no final")
+
+
+def test_prefill_split_invariance_through_state_handoff():
+    """prefill(x[0:T]) == prefill(x[0:T1]) then prefill(x[T1:T]) from the returned state."""
+    tok = make_tokens(200, 2, 4, seed=19, gate_mean=4.0)
+    init = make_state(1, 4, seed=19)
+    full = harness.run_prefill(dict(tokens=tok, cu_seqlens=make_cu_seqlens([200]), initial_state=init))
+    T1 = 90
+    from gdn_inputs import Tokens
+    def part(a, b):
+        return Tokens(q=tok.q[a:b], k=tok.k[a:b], v=tok.v[a:b], g=tok.g[a:b], beta=tok.beta[a:b], Hqk=2, Hv=4, dk=128, dv=128)
+    r1 = harness.run_prefill(dict(tokens=part(0, T1), cu_seqlens=make_cu_seqlens([T1]), initial_state=init))
+    r2 = harness.run_prefill(dict(tokens=part(T1, 200), cu_seqlens=make_cu_seqlens([200 - T1]),
+                                  initial_state=r1["final_state"].astype(np.float32)))
+    assert harness.rel_fro(np.concatenate([r1["out"], r2["out"]]), full["out"]) < 8e-3
+    assert harness.rel_fro(r2["final_state"], full["final_state"]) < 5e-3
+
+
+def test_prefill_long_config_both_initial_states():
+    check(config("prefill_long"), "prefill long zero-init")
+    check(config("prefill_long", initial=True), "prefill long with initial state")
+
+
+def test_prefill_long_weak_decay():
+    check(config("prefill_long", initial=True, gate_mean=6.0), "prefill long weak decay")
+
+
+def test_prefill_varlen_config():
+    check(config("prefill_varlen"), "prefill varlen 16 x U[1,2048]")
