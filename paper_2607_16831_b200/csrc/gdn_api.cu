@@ -1,4 +1,7 @@
 // C-ABI entry points of libgdn: argument validation and launch dispatch only.
+#include <stdio.h>
+#include <stdlib.h>
+
 #include "gdn_common.cuh"
 
 namespace gdn {
@@ -34,6 +37,14 @@ static bool device_supported() {
     return g_device_ok[dev] == 1;
 }
 
+// Maps a CUDA runtime error to a status; with GDN_DEBUG set in the environment the runtime's
+// message goes to stderr (the only case in which the library prints).
+static int cuda_status(cudaError_t e, const char* where) {
+    if (e == cudaSuccess) return GDN_OK;
+    if (getenv("GDN_DEBUG")) fprintf(stderr, "libgdn: %s: %s\n", where, cudaGetErrorString(e));
+    return GDN_ERR_CUDA;
+}
+
 static int check_heads(int Hqk, int Hv, int dk, int dv) {
     if (Hqk <= 0 || Hv <= 0 || dk <= 0 || dv <= 0) return GDN_ERR_SHAPE;
     if (Hv % Hqk != 0) return GDN_ERR_SHAPE;
@@ -53,9 +64,8 @@ static int decode_impl(const void* q, const void* k, const void* v, const float*
         return GDN_ERR_ALIGN;
     if ((long long)B * Hv * 32 > 0x7fffffffLL) return GDN_ERR_SHAPE;
     if (!device_supported()) return GDN_ERR_UNSUPPORTED;
-    cudaError_t e = decode_dispatch(q, k, v, g, beta, state_in, state_out, out, B, Hqk, Hv, variant,
-                                    (cudaStream_t)stream);
-    return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+    return cuda_status(decode_dispatch(q, k, v, g, beta, state_in, state_out, out, B, Hqk, Hv, variant,
+                                       (cudaStream_t)stream), "gdn_decode");
 }
 
 static int check_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
@@ -132,10 +142,9 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
     const size_t need = prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
         return GDN_ERR_WORKSPACE;
-    cudaError_t e = prefill_chunked_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
-                                             total_tokens, num_seqs, max_seqlen, Hqk, Hv, workspace,
-                                             workspace_bytes, (cudaStream_t)stream);
-    return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+    return cuda_status(prefill_chunked_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
+                                                total_tokens, num_seqs, max_seqlen, Hqk, Hv, workspace,
+                                                workspace_bytes, (cudaStream_t)stream), "gdn_prefill");
 }
 
 int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const float* g, const float* beta,
@@ -147,9 +156,9 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const flo
                                num_seqs, max_seqlen, Hqk, Hv, dk, dv, &nothing))
         return rc;
     if (nothing) return GDN_OK;
-    cudaError_t e = prefill_recurrent_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
-                                               total_tokens, num_seqs, Hqk, Hv, (cudaStream_t)stream);
-    return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+    return cuda_status(prefill_recurrent_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
+                                                  total_tokens, num_seqs, Hqk, Hv, (cudaStream_t)stream),
+                       "gdn_prefill_recurrent");
 }
 
 int gdn_last_device_status(void* workspace, int* device_status, void* stream) {

@@ -26,8 +26,19 @@ __device__ __forceinline__ uint16_t float_to_bf16_bits(float x) {
     return __bfloat16_as_ushort(__float2bfloat16_rn(x));
 }
 
+// Two floats -> packed bf16x2 (element 0 in the low half), one conversion instruction.
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    return (uint32_t)float_to_bf16_bits(lo) | ((uint32_t)float_to_bf16_bits(hi) << 16);
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// y0,y1 -> packed bf16 hi parts and packed bf16 of the remainders (y - hi): a two-term
+// bf16 expansion carrying ~16 significant bits.
+__device__ __forceinline__ void split_bf16x2(float y0, float y1, uint32_t& hi, uint32_t& lo) {
+    hi = pack_bf16x2(y0, y1);
+    const float h0 = __uint_as_float(hi << 16), h1 = __uint_as_float(hi & 0xffff0000u);
+    lo = pack_bf16x2(y0 - h0, y1 - h1);
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

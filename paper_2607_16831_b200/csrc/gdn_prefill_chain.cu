@@ -1,0 +1,461 @@
+// Inter-chunk ("chain") kernel of the chunked WY / UT-transform prefill.
+//
+// One CTA per (sequence, value head) walks the sequence's 64-token chunks in order.  With
+// S the fp32 state entering a chunk ([dv][dk], row v = tensor-memory lane v) and the chunk
+// summaries T', W, P and scalars from the intra-chunk kernel:
+//
+//   Delta^T = V^T T'^T - S W^T            [128 x 64]   (G1: T' hi+lo, then G2A on the chain)
+//   Oa^T    = S Q^T                        [128 x 64]   (G2B, off the chain)
+//   Ob^T    = Delta^T P^T                  [128 x 64]   (G3A, off the chain)
+//   S      <- Gamma_L S + (e o Delta)^T K  [128 x 128]  (G3B on the chain, hi+lo)
+//   o_i     = Gamma_i Oa^T[:,i] + Ob^T[:,i]
+//
+// All products are tcgen05.mma with fp32 accumulators in tensor memory.  The operands that
+// the chain itself produces (the bf16 copy of S, Delta^T and its decayed hi/lo copies) are
+// written back to tensor memory and read from there as the A operand, so they never touch
+// shared memory; an MMA's time here is set by the operand bytes it pulls from shared memory,
+// and this halves them.  The B operands are 128-byte-swizzled shared-memory tiles: q/k/v
+// arrive by TMA from the caller's tensors, the chunk summaries by bulk copies of
+// pre-swizzled images, two stages deep.  The fp32 state stays in tensor memory for the
+// whole sequence.  Warp roles:
+//   warps 0-3  chain: drain Delta^T -> bf16 operands; drain S -> bf16 operand + decayed fp32 back
+//   warps 4-7  output: drain Oa/Ob -> bf16 out
+//   warp  8    issues every MMA (one elected lane)
+//   warp  9    issues every TMA / bulk copy, one chunk ahead of the MMAs
+// Hand-offs are mbarriers; every wait is bounded and failure unwinds through an abort flag.
+#include "gdn_prefill_ws.cuh"
+#include "gdn_sm100.cuh"
+
+namespace gdn {
+using namespace sm100;
+
+constexpr int kChainThreads = 320;
+// shared-memory map (bytes from a 1024-byte aligned base): two stages of per-chunk operands
+constexpr uint32_t ST_T = 0;          // T'hi 8K | T'lo 8K   (bulk copy, together with W)
+constexpr uint32_t ST_W = 16384;      // W: 2 tiles [64][64]
+constexpr uint32_t ST_V = 32768;      // V tile: 2 x [64 tokens][64]  (TMA)
+constexpr uint32_t ST_Q = 49152;      // Q tile                        (TMA)
+constexpr uint32_t ST_K = 65536;      // K tile                        (TMA)
+constexpr uint32_t ST_P = 81920;      // P [64][64]                    (bulk copy)
+constexpr uint32_t kStageBytes = 90112;
+constexpr uint32_t OFF_BAR = 2 * kStageBytes;          // mbarriers, TMEM slot, abort flag
+constexpr uint32_t kChainSmem = OFF_BAR + 256 + 1024;  // + slack for the manual 1024-byte alignment
+constexpr uint32_t kTxA = 32768 + 16384 + 16384;       // T'+W, V, Q
+constexpr uint32_t kTxB = 16384 + 8192;                // K, P
+// tensor-memory columns (32-bit each)
+constexpr uint32_t TM_S = 0;        // fp32 state                    128
+constexpr uint32_t TM_DELTA = 128;  // fp32 Delta^T accumulator       64
+constexpr uint32_t TM_OA = 192;     // fp32 S Q^T                     64
+constexpr uint32_t TM_OB = 256;     // fp32 Delta^T P^T               64
+constexpr uint32_t TM_SHI = 320;    // bf16 S      (A operand)        64
+constexpr uint32_t TM_DL = 384;     // bf16 Delta^T (A operand)       32
+constexpr uint32_t TM_DTH = 416;    // bf16 (e o Delta)^T hi          32
+constexpr uint32_t TM_DTL = 448;    // bf16 (e o Delta)^T lo          32
+constexpr uint32_t TM_COLS = 512;
+
+enum { B_FULL_A0 = 0, B_FULL_A1, B_FULL_B0, B_FULL_B1, B_FREE0, B_FREE1, B_DELTA, B_STATE, B_O, B_DW, B_SHI, B_STM, B_OFREE, B_COUNT };
+
+__global__ void __launch_bounds__(kChainThreads, 1)
+gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                         const __grid_constant__ CUtensorMap map_v, const float* initial_state,
+                         uint16_t* __restrict__ out, float* final_state, uint8_t* __restrict__ ws, WsLayout L,
+                         int Hqk, int Hv) {
+    const int h = blockIdx.x % Hv, n = blockIdx.x / Hv;
+    const int hq = h / (Hv / Hqk);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 8 * B_COUNT);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_BAR + 8 * B_COUNT + 8);
+
+    const int* chunk_off = reinterpret_cast<const int*>(ws + L.off_chunk_off);
+    const int4* chunk_info = reinterpret_cast<const int4*>(ws + L.off_chunk_info);
+    const int c_begin = chunk_off[n], c_end = chunk_off[n + 1];
+    const int nchunks = c_end - c_begin;
+
+    if (nchunks <= 0) {  // empty sequence: the state passes through
+        if (final_state && tid < kD) {
+            const size_t sb0 = ((size_t)n * Hv + h) * kD * kD + (size_t)tid * kD;
+            for (int j = 0; j < kD; j += 4) {
+                float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (initial_state) x = *reinterpret_cast<const float4*>(initial_state + sb0 + j);
+                *reinterpret_cast<float4*>(final_state + sb0 + j) = x;
+            }
+        }
+        return;
+    }
+    // chunks of one sequence are consecutive: chunk ci starts at t0_first + 64 ci
+    const int t0_first = chunk_info[c_begin].y;
+    const int t_end = chunk_info[c_end - 1].y + chunk_info[c_end - 1].z;
+
+    if (tid == 0) {
+        for (int i = 0; i < B_COUNT; ++i) {
+            const bool many = (i == B_DW || i == B_SHI || i == B_STM || i == B_OFREE);
+            mbar_init(bars + i, many ? 128u : 1u);
+        }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    if (warp == 8) {
+        __syncwarp();
+        tmem_alloc(tmem_slot, TM_COLS);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    auto scal_ptr = [&](int c) {
+        return reinterpret_cast<const float*>(ws + L.off_scal + ((size_t)c * Hv + h) * kScalBytes);
+    };
+#ifdef GDN_CHAIN_PROFILE
+    // SM-clock stamps of CTA 0 into the unused tail of each chunk's scalar block (4-byte slots from byte 576)
+#define GDN_STAMP(c, slot) do { if (blockIdx.x == 0) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)(c) * Hv + h) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
+#else
+#define GDN_STAMP(c, slot) do { } while (0)
+#endif
+
+    if (warp == 8) {
+        // =========================================================== issuer: MMA
+        // The whole warp runs this loop in lock step; one elected lane issues each MMA.
+        {
+            const uint32_t sb = smem_u32(smem);
+            constexpr uint32_t ID_G1 = umma_idesc_bf16(128, 64, true, false, false);    // V^T (MN-major A) x T'^T
+            constexpr uint32_t ID_G2A = umma_idesc_bf16(128, 64, false, false, true);   // -(S) x W^T
+            constexpr uint32_t ID_N64 = umma_idesc_bf16(128, 64, false, false, false);  // S x Q^T ; Delta^T x P^T
+            constexpr uint32_t ID_G3B = umma_idesc_bf16(128, 128, false, true, false);  // (e o Delta)^T x K (MN-major B)
+            // Shared-memory descriptors are built once (stage 0); the other stage and the K steps only
+            // move the start-address field (16-byte units): +32 B per 16 K-major columns, +2048 B per
+            // 16 MN-major rows, +kStageBytes per stage.
+            constexpr uint64_t kStageStep = kStageBytes >> 4;
+            const uint64_t dV = umma_desc(sb + ST_V, 8192, 1024);
+            const uint64_t dThi = umma_desc(sb + ST_T, 16, 1024), dTlo = umma_desc(sb + ST_T + 8192, 16, 1024);
+            const uint64_t dW0 = umma_desc(sb + ST_W, 16, 1024), dW1 = umma_desc(sb + ST_W + 8192, 16, 1024);
+            const uint64_t dQ0 = umma_desc(sb + ST_Q, 16, 1024), dQ1 = umma_desc(sb + ST_Q + 8192, 16, 1024);
+            const uint64_t dK = umma_desc(sb + ST_K, 8192, 1024), dP = umma_desc(sb + ST_P, 16, 1024);
+            auto issue_G1 = [&](int st) {
+                const uint64_t so = st * kStageStep;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_bf16_ss_warp(tmem_base + TM_DELTA, dV + so + ks * 128, dThi + so + ks * 2, ID_G1, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_bf16_ss_warp(tmem_base + TM_DELTA, dV + so + ks * 128, dTlo + so + ks * 2, ID_G1, 1);
+            };
+
+            bool g1_issued = false;
+
+#define GDN_WAIT(idx, parity) if (!mbar_wait_all(bars + (idx), (uint32_t)(parity), abort_flag)) break
+
+            for (int ci = 0; ci < nchunks; ++ci) {
+                const int c = c_begin + ci;
+                (void)c;
+                const int st = ci & 1, par = ci & 1, ph2 = (ci >> 1) & 1;
+                const uint64_t so = st * kStageStep;
+                const bool last = (ci + 1 == nchunks);
+                if (lane == 0) GDN_STAMP(c, 0);
+                if (!g1_issued) {
+                    GDN_WAIT(B_FULL_A0 + st, ph2);
+                    tc_fence_after_sync();
+                    issue_G1(st);
+                }
+                g1_issued = false;
+                // ---- on the chain: Delta^T -= S W^T   (A = bf16 S in tensor memory)
+                GDN_WAIT(B_SHI, par);
+                if (lane == 0) GDN_STAMP(c, 2);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    umma_bf16_ts_warp(tmem_base + TM_DELTA, tmem_base + TM_SHI + ks * 8,
+                                 (ks < 4 ? dW0 : dW1) + so + (ks & 3) * 2, ID_G2A, 1);
+                umma_commit_warp(bars + B_DELTA);
+                if (lane == 0) GDN_STAMP(c, 4);
+                // ---- off the chain: Oa^T = S Q^T (runs while the chain warps drain Delta^T)
+                if (ci >= 1) GDN_WAIT(B_OFREE, par ^ 1);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    umma_bf16_ts_warp(tmem_base + TM_OA, tmem_base + TM_SHI + ks * 8,
+                                 (ks < 4 ? dQ0 : dQ1) + so + (ks & 3) * 2, ID_N64, ks > 0);
+                if (lane == 0) GDN_STAMP(c, 5);
+                // ---- on the chain: S += (e o Delta)^T K  (hi + lo; A in tensor memory, B = K MN-major)
+                GDN_WAIT(B_FULL_B0 + st, ph2);
+                GDN_WAIT(B_STM, par);
+                if (lane == 0) GDN_STAMP(c, 7);
+                GDN_WAIT(B_DW, par);
+                if (lane == 0) GDN_STAMP(c, 8);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_bf16_ts_warp(tmem_base + TM_S, tmem_base + TM_DTH + ks * 8, dK + so + ks * 128, ID_G3B, 1);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_bf16_ts_warp(tmem_base + TM_S, tmem_base + TM_DTL + ks * 8, dK + so + ks * 128, ID_G3B, 1);
+                umma_commit_warp(bars + B_STATE);
+                if (lane == 0) GDN_STAMP(c, 9);
+                // ---- off the chain: Ob^T = Delta^T P^T, and the next chunk's V^T T'^T if it has landed
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_bf16_ts_warp(tmem_base + TM_OB, tmem_base + TM_DL + ks * 8, dP + so + ks * 2, ID_N64, ks > 0);
+                if (!last && __shfl_sync(0xffffffffu, lane == 0 ? (uint32_t)mbar_try_wait(bars + B_FULL_A0 + (st ^ 1), ((ci + 1) >> 1) & 1) : 0u, 0)) {
+                    tc_fence_after_sync();
+                    issue_G1(st ^ 1);
+                    g1_issued = true;
+                }
+                umma_commit_warp(bars + B_O);
+                umma_commit_warp(bars + B_FREE0 + st);  // every MMA that reads this stage has been issued
+                if (lane == 0) GDN_STAMP(c, 10);
+            }
+#undef GDN_WAIT
+        }
+        __syncwarp();
+    } else if (warp == 9) {
+        // =========================================================== producer: all TMA / bulk copies
+        {
+            if (lane == 0) {
+                prefetch_tensormap(&map_q);
+                prefetch_tensormap(&map_k);
+                prefetch_tensormap(&map_v);
+            }
+            __syncwarp();
+            auto load_all = [&](int c, int st) {
+                if (!elect_one()) return;
+                uint8_t* sp = smem + st * kStageBytes;
+                const int t0 = t0_first + (c - c_begin) * kChunk;
+                mbar_expect_tx(bars + B_FULL_A0 + st, kTxA);
+                bulk_load(sp + ST_T, ws + L.off_A + ((size_t)c * Hv + h) * kABytes, kABytes, bars + B_FULL_A0 + st);
+                tma_load_3d(sp + ST_V, &map_v, bars + B_FULL_A0 + st, 0, h, t0);
+                tma_load_3d(sp + ST_V + 8192, &map_v, bars + B_FULL_A0 + st, 64, h, t0);
+                tma_load_3d(sp + ST_Q, &map_q, bars + B_FULL_A0 + st, 0, hq, t0);
+                tma_load_3d(sp + ST_Q + 8192, &map_q, bars + B_FULL_A0 + st, 64, hq, t0);
+                mbar_expect_tx(bars + B_FULL_B0 + st, kTxB);
+                tma_load_3d(sp + ST_K, &map_k, bars + B_FULL_B0 + st, 0, hq, t0);
+                tma_load_3d(sp + ST_K + 8192, &map_k, bars + B_FULL_B0 + st, 64, hq, t0);
+                bulk_load(sp + ST_P, ws + L.off_P + ((size_t)c * Hv + h) * kPBytes, kPBytes, bars + B_FULL_B0 + st);
+            };
+            // chunk ci goes to stage ci & 1 as soon as the MMAs of chunk ci - 2 have drained it
+            for (int ci = 0; ci < nchunks; ++ci) {
+                if (ci >= 2 &&
+                    !mbar_wait_all(bars + B_FREE0 + (ci & 1), (uint32_t)(((ci >> 1) - 1) & 1), abort_flag))
+                    break;
+                load_all(c_begin + ci, ci & 1);
+            }
+        }
+        __syncwarp();
+    } else if (warp < 4) {
+        // =========================================================== chain warps
+        const int v = tid;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
+        const size_t sbase = ((size_t)n * Hv + h) * kD * kD + (size_t)v * kD;
+        // initial state: bf16 operand copy and Gamma_L(first chunk) * S, both into tensor memory
+        {
+            const float gl0 = __ldg(scal_ptr(c_begin) + 128);
+#pragma unroll 1
+            for (int b = 0; b < 2; ++b) {
+                uint32_t r0[32], r1[32], pk[32];
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
+                    if (initial_state) {
+                        x = *reinterpret_cast<const float4*>(initial_state + sbase + b * 64 + j);
+                        y = *reinterpret_cast<const float4*>(initial_state + sbase + b * 64 + 32 + j);
+                    }
+                    r0[j + 0] = __float_as_uint(x.x); r0[j + 1] = __float_as_uint(x.y);
+                    r0[j + 2] = __float_as_uint(x.z); r0[j + 3] = __float_as_uint(x.w);
+                    r1[j + 0] = __float_as_uint(y.x); r1[j + 1] = __float_as_uint(y.y);
+                    r1[j + 2] = __float_as_uint(y.z); r1[j + 3] = __float_as_uint(y.w);
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    pk[j] = pack_bf16x2(__uint_as_float(r0[2 * j]), __uint_as_float(r0[2 * j + 1]));
+                    pk[16 + j] = pack_bf16x2(__uint_as_float(r1[2 * j]), __uint_as_float(r1[2 * j + 1]));
+                }
+                tmem_st32(lane_addr + TM_SHI + b * 32, pk);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    r0[j] = __float_as_uint(__uint_as_float(r0[j]) * gl0);
+                    r1[j] = __float_as_uint(__uint_as_float(r1[j]) * gl0);
+                }
+                tmem_st32(lane_addr + TM_S + b * 64, r0);
+                tmem_st32(lane_addr + TM_S + b * 64 + 32, r1);
+            }
+            tmem_st_wait();
+            tc_fence_before_sync();
+            mbar_arrive(bars + B_SHI);
+            mbar_arrive(bars + B_STM);
+        }
+        for (int ci = 0; ci < nchunks; ++ci) {
+            const int c = c_begin + ci;
+            const uint32_t par = ci & 1;
+            const bool last = (ci + 1 == nchunks);
+            const float gl_next = last ? 1.f : __ldg(scal_ptr(c + 1) + 128);
+            // e_j of this chunk into registers before the wait; prefetch the next chunk's lines
+            float4 ev4[16];
+            {
+                const float4* e4 = reinterpret_cast<const float4*>(scal_ptr(c) + 64);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) ev4[j] = __ldg(e4 + j);
+                if (!last) asm volatile("prefetch.global.L2 [%0];" ::"l"(scal_ptr(c + 1) + (lane & 3) * 32));
+            }
+            if (tid == 0) GDN_STAMP(c, 16);
+            if (!mbar_wait_all(bars + B_DELTA, par, abort_flag)) break;
+            tc_fence_after_sync();
+            if (tid == 0) GDN_STAMP(c, 17);
+            // Delta^T row v -> bf16 A operands in tensor memory: Delta, and (e o Delta) as hi + lo.
+            // Two halves of 32 tokens keep the live registers low (9 warps share the register file).
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t r[32], xd[16], hd[16], ld[16];
+                tmem_ld32(lane_addr + TM_DELTA + half * 32, r);
+                tmem_ld_wait();
+                if (tid == 0 && half == 0) GDN_STAMP(c, 28);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float4 ea = ev4[half * 8 + (j >> 1)];
+                    const float e0 = (j & 1) ? ea.z : ea.x, e1 = (j & 1) ? ea.w : ea.y;
+                    const float x0 = __uint_as_float(r[2 * j]), x1 = __uint_as_float(r[2 * j + 1]);
+                    xd[j] = pack_bf16x2(x0, x1);
+                    split_bf16x2(x0 * e0, x1 * e1, hd[j], ld[j]);
+                }
+                tmem_st16(lane_addr + TM_DTH + half * 16, hd);
+                tmem_st16(lane_addr + TM_DTL + half * 16, ld);
+                tmem_st16(lane_addr + TM_DL + half * 16, xd);
+            }
+            tmem_st_wait();
+            tc_fence_before_sync();
+            mbar_arrive(bars + B_DW);
+            if (tid == 0) GDN_STAMP(c, 18);
+
+            if (!mbar_wait_all(bars + B_STATE, par, abort_flag)) break;
+            tc_fence_after_sync();
+            if (tid == 0) GDN_STAMP(c, 19);
+            if (last) {
+                if (final_state) {
+#pragma unroll 1
+                    for (int b = 0; b < 4; ++b) {
+                        uint32_t r[32];
+                        tmem_ld32(lane_addr + TM_S + b * 32, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<float4*>(final_state + sbase + b * 32 + j) = make_float4(
+                                __uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                    }
+                }
+            } else {
+                // state row v: bf16 operand copy for the next chunk first (it gates the next G2A) ...
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    uint32_t r0[32], r1[32], pk[32];
+                    tmem_ld32(lane_addr + TM_S + b * 64, r0);
+                    tmem_ld32(lane_addr + TM_S + b * 64 + 32, r1);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        pk[j] = pack_bf16x2(__uint_as_float(r0[2 * j]), __uint_as_float(r0[2 * j + 1]));
+                        pk[16 + j] = pack_bf16x2(__uint_as_float(r1[2 * j]), __uint_as_float(r1[2 * j + 1]));
+                    }
+                    tmem_st32(lane_addr + TM_SHI + b * 32, pk);
+                }
+                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(bars + B_SHI);
+                if (tid == 0) GDN_STAMP(c, 20);
+                // ... then the fp32 state decayed by the next chunk's Gamma_L, in place (gates the next G3B)
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    uint32_t r0[32], r1[32];
+                    tmem_ld32(lane_addr + TM_S + b * 64, r0);
+                    tmem_ld32(lane_addr + TM_S + b * 64 + 32, r1);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        r0[j] = __float_as_uint(__uint_as_float(r0[j]) * gl_next);
+                        r1[j] = __float_as_uint(__uint_as_float(r1[j]) * gl_next);
+                    }
+                    tmem_st32(lane_addr + TM_S + b * 64, r0);
+                    tmem_st32(lane_addr + TM_S + b * 64 + 32, r1);
+                }
+                tmem_st_wait();
+                tc_fence_before_sync();
+                mbar_arrive(bars + B_STM);
+                if (tid == 0) GDN_STAMP(c, 21);
+            }
+        }
+    } else {
+        // =========================================================== output warps
+        const int v = tid - 128;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+        for (int ci = 0; ci < nchunks; ++ci) {
+            const int c = c_begin + ci;
+            const uint32_t par = ci & 1;
+            const int t0 = t0_first + ci * kChunk, len = min(kChunk, t_end - t0);
+            auto last_chunk = [&](int i) { return i + 1 == nchunks; };
+            const float4* g4 = reinterpret_cast<const float4*>(scal_ptr(c));  // Gamma_i of this chunk
+            if (!last_chunk(ci)) asm volatile("prefetch.global.L2 [%0];" ::"l"(scal_ptr(c + 1) + (lane & 1) * 32));
+            if (tid == 128) GDN_STAMP(c, 24);
+            if (!mbar_wait_all(bars + B_O, par, abort_flag)) break;
+            tc_fence_after_sync();
+            if (tid == 128) GDN_STAMP(c, 25);
+            // o_i = Gamma_i Oa^T[v][i] + Ob^T[v][i], packed two tokens per register
+            uint32_t op[32];
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t a[32], b[32];
+                tmem_ld32(lane_addr + TM_OA + half * 32, a);
+                tmem_ld32(lane_addr + TM_OB + half * 32, b);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j4 = 0; j4 < 8; ++j4) {
+                    const float4 gm = __ldg(g4 + half * 8 + j4);
+                    op[half * 16 + j4 * 2] = pack_bf16x2(fmaf(gm.x, __uint_as_float(a[4 * j4]), __uint_as_float(b[4 * j4])),
+                                                         fmaf(gm.y, __uint_as_float(a[4 * j4 + 1]), __uint_as_float(b[4 * j4 + 1])));
+                    op[half * 16 + j4 * 2 + 1] = pack_bf16x2(fmaf(gm.z, __uint_as_float(a[4 * j4 + 2]), __uint_as_float(b[4 * j4 + 2])),
+                                                             fmaf(gm.w, __uint_as_float(a[4 * j4 + 3]), __uint_as_float(b[4 * j4 + 3])));
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(bars + B_OFREE);
+            if (tid == 128) GDN_STAMP(c, 26);
+            uint16_t* orow = out + ((size_t)t0 * Hv + h) * kD + v;
+            const size_t ostride = (size_t)Hv * kD;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                if (2 * j < len) orow[(size_t)(2 * j) * ostride] = (uint16_t)(op[j] & 0xffffu);
+                if (2 * j + 1 < len) orow[(size_t)(2 * j + 1) * ostride] = (uint16_t)(op[j] >> 16);
+            }
+            if (tid == 128) GDN_STAMP(c, 27);
+        }
+    }
+
+    // ---- unwind: on failure give copies in flight a moment to land, then release tensor memory
+    if (*abort_flag) {
+        const long long t_start = clock64();
+        while (clock64() - t_start < 400000) { }
+        if (tid == 0) atomicExch(reinterpret_cast<int*>(ws), kStatusTimeout);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 8) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, TM_COLS);
+    }
+}
+
+cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                                 const float* initial_state, void* out, float* final_state, uint8_t* ws,
+                                 const WsLayout& L, int num_seqs, int Hqk, int Hv, cudaStream_t st) {
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(gdn_prefill_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kChainSmem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    gdn_prefill_chain_kernel<<<(unsigned)((long long)num_seqs * Hv), kChainThreads, kChainSmem, st>>>(
+        mq, mk, mv, initial_state, (uint16_t*)out, final_state, ws, L, Hqk, Hv);
+    return cudaGetLastError();
+}
+
+}  // namespace gdn

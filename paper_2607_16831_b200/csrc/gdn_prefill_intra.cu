@@ -1,0 +1,351 @@
+// Chunk table and intra-chunk kernel of the chunked WY / UT-transform prefill.
+//
+// Per (chunk, value head), with gamma the cumulative log-gate inside the chunk,
+// Gamma = exp(gamma), D_ij = exp(gamma_i - gamma_j) for j <= i:
+//   A  = strict_lower(diag(beta) (K K^T o D))     the kk^T lower-triangular system
+//   T  = (I + A)^-1                               UT transform by substitution (fp32)
+//   T' = T diag(beta)   (bf16 hi + lo),   W = T' diag(Gamma) K,   P = (Q K^T) o D
+// K K^T, Q K^T and W run on tcgen05 (bf16 operands fed by TMA, fp32 accumulation); the gate
+// algebra and the triangular solve stay in fp32 registers.
+// and the per-token scalars Gamma_i, e_i = exp(gamma_L - gamma_i), Gamma_L.  Everything is
+// written to the workspace already in the 128-byte-swizzled shared-memory image that the
+// chain kernel hands to the tensor cores.
+#include "gdn_prefill_ws.cuh"
+#include "gdn_sm100.cuh"
+
+namespace gdn {
+using namespace sm100;
+
+// ------------------------------------------------------------------ prep: chunk table
+__global__ void __launch_bounds__(256)
+gdn_prefill_prep_kernel(const int32_t* __restrict__ cu, int num_seqs, int total_tokens, int* hdr,
+                        int* chunk_off, int4* chunk_info, int nc_max) {
+    __shared__ int part[257];
+    const int tid = threadIdx.x;
+    const int per = (num_seqs + 255) / 256;
+    const int lo = min(num_seqs, tid * per), hi = min(num_seqs, lo + per);
+    int sum = 0;
+    for (int n = lo; n < hi; ++n) {
+        const int t0 = max(0, min(cu[n], total_tokens));
+        const int t1 = max(t0, min(cu[n + 1], total_tokens));
+        sum += (t1 - t0 + kChunk - 1) / kChunk;
+    }
+    part[tid] = sum;
+    __syncthreads();
+    if (tid == 0) {
+        int run = 0;
+        for (int i = 0; i < 256; ++i) {
+            const int t = part[i];
+            part[i] = run;
+            run += t;
+        }
+        part[256] = run;
+        hdr[0] = 0;
+        hdr[1] = min(run, nc_max);
+        chunk_off[num_seqs] = min(run, nc_max);
+    }
+    __syncthreads();
+    int base = part[tid];
+    for (int n = lo; n < hi; ++n) {
+        const int t0 = max(0, min(cu[n], total_tokens));
+        const int t1 = max(t0, min(cu[n + 1], total_tokens));
+        const int nch = (t1 - t0 + kChunk - 1) / kChunk;
+        chunk_off[n] = min(base, nc_max);
+        for (int j = 0; j < nch; ++j)
+            if (base + j < nc_max) chunk_info[base + j] = make_int4(n, t0 + j * kChunk, min(kChunk, t1 - t0 - j * kChunk), j);
+        base += nch;
+    }
+}
+
+// ------------------------------------------------------------------ intra-chunk kernel
+// One CTA (128 threads) per (chunk, q/k head); the G value heads that share the q/k head are
+// processed in pairs so that every tensor-core product has M = 128:
+//   MMA1  [Q ; K] K^T            (128 x 64 x 128)  rows 0-63: Q K^T, rows 64-127: K K^T
+//   solve T = (I + A)^-1         fp32, one thread per ROW of T through the transposed system
+//                                y (I + A) = e_i  (backward substitution over columns)
+//   MMA2  [T''_a ; T''_b] K      (128 x 128 x 64)  T'' = T diag(beta o Gamma), bf16 hi + lo
+constexpr int kIntraThreads = 128;
+constexpr uint32_t IQ_LO = 0, IK_LO = 8192, IQ_HI = 16384, IK_HI = 24576;  // TMA tiles [64][64] bf16
+constexpr uint32_t IT2 = 32768;      // T'' operand: hi [128][64] 16 KB | lo 16 KB
+constexpr uint32_t IAT = 65536;      // A^T for two heads, fp32 [2][64][kATP]
+constexpr int kATP = 68;
+constexpr uint32_t IGAM = IAT + 2 * 64 * kATP * 4;  // gam[2][64] | bet[2][64] | Gam[2][64] | tmp[4]
+constexpr uint32_t IBAR = IGAM + 6 * 64 * 4 + 64;
+constexpr uint32_t kIntraSmem = IBAR + 64 + 1024;
+constexpr uint32_t ITM_D1 = 0, ITM_D2 = 64, ITM_COLS = 256;
+
+__global__ void __launch_bounds__(kIntraThreads)
+gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                         const float* __restrict__ g, const float* __restrict__ beta, uint8_t* __restrict__ ws,
+                         WsLayout L, int Hqk, int Hv) {
+    const int c = blockIdx.x, hq = blockIdx.y;
+    const int* hdr = reinterpret_cast<const int*>(ws);
+    if (c >= hdr[1]) return;
+    const int4 info = reinterpret_cast<const int4*>(ws + L.off_chunk_info)[c];
+    const int t0 = info.y, len = info.z;
+    const int G = Hv / Hqk;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int hh = tid >> 6, i = tid & 63;  // role in the gate / solve / W phases: head of the pair, row
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    float* At = reinterpret_cast<float*>(smem + IAT);
+    float* gam = reinterpret_cast<float*>(smem + IGAM);
+    float* bet = gam + 128;
+    float* Gam = gam + 256;
+    float* tmp = gam + 384;
+    uint64_t* bar_load = reinterpret_cast<uint64_t*>(smem + IBAR);
+    uint64_t* bar_mma1 = bar_load + 1;
+    uint64_t* bar_mma2 = bar_load + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + IBAR + 32);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + IBAR + 40);
+
+    if (tid == 0) {
+        mbar_init(bar_load, 1);
+        mbar_init(bar_mma1, 1);
+        mbar_init(bar_mma2, 1);
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc(tmem_slot, ITM_COLS);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const uint32_t sb = smem_u32(smem);
+    bool ok = true;
+
+    if (warp == 0) {
+        if (elect_one()) {
+            prefetch_tensormap(&map_q);
+            prefetch_tensormap(&map_k);
+            mbar_expect_tx(bar_load, 32768);
+            tma_load_3d(smem + IQ_LO, &map_q, bar_load, 0, hq, t0);
+            tma_load_3d(smem + IQ_HI, &map_q, bar_load, 64, hq, t0);
+            tma_load_3d(smem + IK_LO, &map_k, bar_load, 0, hq, t0);
+            tma_load_3d(smem + IK_HI, &map_k, bar_load, 64, hq, t0);
+        }
+        __syncwarp();
+        ok = mbar_wait_all(bar_load, 0, abort_flag);
+        if (ok) {
+            tc_fence_after_sync();
+            constexpr uint32_t ID1 = umma_idesc_bf16(128, 64, false, false, false);
+            const uint64_t dA0 = umma_desc(sb + IQ_LO, 16, 1024), dA1 = umma_desc(sb + IQ_HI, 16, 1024);
+            const uint64_t dB0 = umma_desc(sb + IK_LO, 16, 1024), dB1 = umma_desc(sb + IK_HI, 16, 1024);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) umma_bf16_ss_warp(tmem_base + ITM_D1, dA0 + ks * 2, dB0 + ks * 2, ID1, ks > 0);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) umma_bf16_ss_warp(tmem_base + ITM_D1, dA1 + ks * 2, dB1 + ks * 2, ID1, 1);
+            umma_commit_warp(bar_mma1);
+        }
+    }
+
+    ok = __syncthreads_and(ok);  // uniform across the CTA: nobody enters the loop if the load gave up
+
+    const int npairs = (G + 1) / 2;
+    for (int p = 0; p < npairs && ok; ++p) {
+        const int nh = min(2, G - 2 * p);
+        const int h = hq * G + 2 * p + hh;  // this thread's value head in the gate / solve / W phases
+        const bool head_ok = hh < nh;
+        // ---- gates of both heads: gamma = inclusive cumsum of g (fp32), beta; zero beyond len
+        {
+            float x = 0.f, b = 0.f;
+            if (head_ok && i < len) {
+                x = __ldg(g + (size_t)(t0 + i) * Hv + h);
+                b = __ldg(beta + (size_t)(t0 + i) * Hv + h);
+            }
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const float y = __shfl_up_sync(0xffffffffu, x, o);
+                if (lane >= o) x += y;
+            }
+            if ((warp & 1) == 0 && lane == 31) tmp[hh] = x;
+            __syncthreads();
+            if (warp & 1) x += tmp[hh];
+            gam[tid] = x;
+            bet[tid] = b;
+            Gam[tid] = __expf(x);
+            __syncthreads();
+        }
+        if (p == 0) {
+            ok = mbar_wait_all(bar_mma1, 0, abort_flag);
+            ok = __syncthreads_and(ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+        }
+        // ---- phase A: this thread's row of [Q K^T ; K K^T]: rows 0-63 -> P, rows 64-127 -> A^T
+        {
+            uint32_t r0[32], r1[32];
+            tmem_ld32(lane_addr + ITM_D1, r0);
+            tmem_ld32(lane_addr + ITM_D1 + 32, r1);
+            tmem_ld_wait();
+            const int row = tid & 63;
+            for (int e = 0; e < nh; ++e) {
+                const float* gm = gam + e * 64;
+                const float gi = gm[row];
+                const int hv = hq * G + 2 * p + e;
+                if (tid < 64) {
+                    // P row: (Q K^T)_ij exp(gamma_i - gamma_j) for j <= i (difference masked before exp)
+                    uint8_t* wsP = ws + L.off_P + ((size_t)c * Hv + hv) * kPBytes;
+#pragma unroll
+                    for (int c16 = 0; c16 < 8; ++c16) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int q2 = 0; q2 < 4; ++q2) {
+                            const int j = c16 * 8 + q2 * 2;
+                            const float a0 = __uint_as_float(j < 32 ? r0[j] : r1[j - 32]);
+                            const float a1 = __uint_as_float(j + 1 < 32 ? r0[j + 1] : r1[j + 1 - 32]);
+                            const float p0 = (j <= row && row < len) ? a0 * __expf(gi - gm[j]) : 0.f;
+                            const float p1 = (j + 1 <= row && row < len) ? a1 * __expf(gi - gm[j + 1]) : 0.f;
+                            pk[q2] = pack_bf16x2(p0, p1);
+                        }
+                        *reinterpret_cast<uint4*>(wsP + swz(row, c16)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                } else {
+                    // A^T[j][i] = beta_i exp(gamma_i - gamma_j) (K K^T)_ij for j < i, else 0
+                    float* at = At + e * 64 * kATP;
+                    const float bi = bet[e * 64 + row];
+#pragma unroll
+                    for (int j = 0; j < 64; ++j) {
+                        const float a = __uint_as_float(j < 32 ? r0[j] : r1[j - 32]);
+                        at[j * kATP + row] = (j < row) ? bi * __expf(gi - gm[j]) * a : 0.f;
+                    }
+                }
+            }
+        }
+        // per-token scalars of this thread's (head, row)
+        if (head_ok) {
+            float* wsS = reinterpret_cast<float*>(ws + L.off_scal + ((size_t)c * Hv + h) * kScalBytes);
+            wsS[i] = Gam[tid];
+            wsS[64 + i] = __expf(gam[hh * 64 + len - 1] - gam[tid]);
+            if (i == 0) wsS[128] = Gam[hh * 64 + len - 1];
+        }
+        __syncthreads();
+        // ---- UT transform, row i of T = (I + A)^-1:  y_j = delta_ij - sum_{m > j} y_m A[m][j]
+        float y[64];
+#pragma unroll
+        for (int j = 0; j < 64; ++j) y[j] = (j == i) ? 1.f : 0.f;
+        {
+            const float* at = At + hh * 64 * kATP;
+#pragma unroll
+            for (int j = 62; j >= 0; --j) {
+                float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+                const float* arow = at + j * kATP;
+                // m runs over (j, 63]; float4 groups that start above j
+                const int m0 = (j + 1 + 3) & ~3;
+#pragma unroll
+                for (int m = j + 1; m < m0 && m < 64; ++m) acc0 = fmaf(arow[m], y[m], acc0);
+#pragma unroll
+                for (int m = m0; m < 64; m += 4) {
+                    const float4 a4 = *reinterpret_cast<const float4*>(arow + m);
+                    acc0 = fmaf(a4.x, y[m], acc0);
+                    acc1 = fmaf(a4.y, y[m + 1], acc1);
+                    acc2 = fmaf(a4.z, y[m + 2], acc2);
+                    acc3 = fmaf(a4.w, y[m + 3], acc3);
+                }
+                y[j] -= (acc0 + acc1) + (acc2 + acc3);
+            }
+        }
+        // ---- T' = T diag(beta) -> workspace (bf16 hi + lo); T'' = T' diag(Gamma) -> smem A operand (hi + lo)
+        {
+            uint8_t* wsA = ws + L.off_A + ((size_t)c * Hv + h) * kABytes;
+            const float* bt = bet + hh * 64;
+            const float* Gm = Gam + hh * 64;
+#pragma unroll
+            for (int c16 = 0; c16 < 8; ++c16) {
+                uint32_t h1[4], l1[4], h2[4], l2[4];
+#pragma unroll
+                for (int q2 = 0; q2 < 4; ++q2) {
+                    const int j = c16 * 8 + q2 * 2;
+                    const float a0 = y[j] * bt[j], a1 = y[j + 1] * bt[j + 1];
+                    split_bf16x2(a0, a1, h1[q2], l1[q2]);
+                    split_bf16x2(a0 * Gm[j], a1 * Gm[j + 1], h2[q2], l2[q2]);
+                }
+                if (head_ok) {
+                    *reinterpret_cast<uint4*>(wsA + swz(i, c16)) = make_uint4(h1[0], h1[1], h1[2], h1[3]);
+                    *reinterpret_cast<uint4*>(wsA + 8192 + swz(i, c16)) = make_uint4(l1[0], l1[1], l1[2], l1[3]);
+                }
+                *reinterpret_cast<uint4*>(smem + IT2 + swz(tid, c16)) = make_uint4(h2[0], h2[1], h2[2], h2[3]);
+                *reinterpret_cast<uint4*>(smem + IT2 + 16384 + swz(tid, c16)) = make_uint4(l2[0], l2[1], l2[2], l2[3]);
+            }
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        __syncthreads();
+        // ---- MMA2: W (both heads) = [T''_a ; T''_b] K, K read MN-major from the TMA tiles
+        if (warp == 0) {
+            tc_fence_after_sync();
+            constexpr uint32_t ID2 = umma_idesc_bf16(128, 128, false, true, false);
+            const uint64_t dTh = umma_desc(sb + IT2, 16, 1024), dTl = umma_desc(sb + IT2 + 16384, 16, 1024);
+            const uint64_t dK = umma_desc(sb + IK_LO, IK_HI - IK_LO, 1024);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) umma_bf16_ss_warp(tmem_base + ITM_D2, dTh + ks * 2, dK + ks * 128, ID2, ks > 0);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) umma_bf16_ss_warp(tmem_base + ITM_D2, dTl + ks * 2, dK + ks * 128, ID2, 1);
+            umma_commit_warp(bar_mma2);
+        }
+        ok = mbar_wait_all(bar_mma2, (uint32_t)(p & 1), abort_flag);
+        ok = __syncthreads_and(ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+        // ---- W row i of head h -> workspace (K-major B operand image: two [64][64] tiles)
+        {
+            uint8_t* wsW = ws + L.off_A + ((size_t)c * Hv + h) * kABytes + 16384;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                uint32_t r[32];
+                tmem_ld32(lane_addr + ITM_D2 + b * 32, r);
+                tmem_ld_wait();
+                if (head_ok) {
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) {
+                        uint4 o;
+                        o.x = pack_bf16x2(__uint_as_float(r[cc * 8 + 0]), __uint_as_float(r[cc * 8 + 1]));
+                        o.y = pack_bf16x2(__uint_as_float(r[cc * 8 + 2]), __uint_as_float(r[cc * 8 + 3]));
+                        o.z = pack_bf16x2(__uint_as_float(r[cc * 8 + 4]), __uint_as_float(r[cc * 8 + 5]));
+                        o.w = pack_bf16x2(__uint_as_float(r[cc * 8 + 6]), __uint_as_float(r[cc * 8 + 7]));
+                        *reinterpret_cast<uint4*>(wsW + (b >> 1) * 8192 + swz(i, (b & 1) * 4 + cc)) = o;
+                    }
+                }
+            }
+        }
+        tc_fence_before_sync();
+        __syncthreads();  // the next pair reuses A^T, the T'' tiles and the W accumulator
+    }
+
+    if (*abort_flag && tid == 0) atomicExch(reinterpret_cast<int*>(ws), kStatusTimeout);
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, ITM_COLS);
+    }
+}
+
+cudaError_t launch_prefill_prep(const int32_t* cu_seqlens, int num_seqs, int total_tokens, uint8_t* ws,
+                                const WsLayout& L, cudaStream_t st) {
+    gdn_prefill_prep_kernel<<<1, 256, 0, st>>>(cu_seqlens, num_seqs, total_tokens, reinterpret_cast<int*>(ws),
+                                               reinterpret_cast<int*>(ws + L.off_chunk_off),
+                                               reinterpret_cast<int4*>(ws + L.off_chunk_info), L.nc_max);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, const float* g, const float* beta,
+                                 uint8_t* ws, const WsLayout& L, int Hqk, int Hv, cudaStream_t st) {
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(gdn_prefill_intra_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kIntraSmem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    dim3 grid(L.nc_max, Hqk);
+    gdn_prefill_intra_kernel<<<grid, kIntraThreads, kIntraSmem, st>>>(mq, mk, g, beta, ws, L, Hqk, Hv);
+    return cudaGetLastError();
+}
+
+}  // namespace gdn

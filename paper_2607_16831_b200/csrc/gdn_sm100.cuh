@@ -27,15 +27,28 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+// One poll.  The thread may be suspended by the hardware for up to `hint_ns` nanoseconds
+// while the phase is incomplete (it wakes as soon as the phase completes), which keeps
+// waiting warps out of the shared-memory pipeline instead of hammering it with polls.
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint_ns = 0) {
     uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
+    if (hint_ns == 0) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+            : "memory");
+    }
     return ok != 0;
 }
 // Bounded wait: gives up after about `limit_cycles` SM clocks (default ~1 s), or as soon
@@ -45,15 +58,46 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
                                           long long limit_cycles = 2000000000LL) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
+#ifndef GDN_WAIT_MODE
+#define GDN_WAIT_MODE 1
+#endif
     for (uint32_t i = 1;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 31u) == 0u) {
+#if GDN_WAIT_MODE == 0
+        if (mbar_try_wait(bar, parity)) return true;             // plain polling
+        if ((i & 63u) == 0u) {
             if (*abort) return false;
             if (clock64() - start > limit_cycles) break;
         }
+#elif GDN_WAIT_MODE == 1
+        if (mbar_try_wait(bar, parity, 20000u)) return true;     // sleeps up to 20 us per poll
+        if (*abort) return false;
+        if (clock64() - start > limit_cycles) break;
+#else
+        if (mbar_try_wait(bar, parity)) return true;             // polling with a short back-off
+        __nanosleep(40);
+        if ((i & 15u) == 0u) {
+            if (*abort) return false;
+            if (clock64() - start > limit_cycles) break;
+        }
+#endif
     }
     *abort = 1;
     return false;
+}
+
+// Warp-collective bounded wait: lane 0 polls and the result is broadcast.  Thirty-two lanes
+// polling the same mbarrier are served one after the other by the shared-memory pipe (about
+// 250 clocks per wait even when the phase is already complete); one poller costs ~30.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort,
+                                               long long limit_cycles = 2000000000LL) {
+    uint32_t ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort, limit_cycles) ? 1u : 0u;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+// Every lane polls; the warp proceeds only if all lanes saw the phase complete.
+__device__ __forceinline__ bool mbar_wait_all(uint64_t* bar, uint32_t parity, volatile int* abort,
+                                              long long limit_cycles = 2000000000LL) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort, limit_cycles));
 }
 
 // ---------------------------------------------------------------- fences
@@ -124,6 +168,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
           "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // ---------------------------------------------------------------- UMMA descriptors
@@ -161,6 +212,54 @@ __device__ __forceinline__ void umma_bf16_ss(uint32_t d_tmem, uint64_t a_desc, u
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Same with the A operand read from tensor memory (row m in lane m, two bf16 per 32-bit
+// column, K along the columns); A must be K-major.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Warp-collective forms: every lane of a converged warp executes the call with identical
+// arguments and one elected lane issues.  Keeping the surrounding code warp-uniform lets the
+// compiler hold descriptors and addresses in uniform registers, which makes an MMA issue
+// several times cheaper than issuing from inside an `if (lane == 0)` branch.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred px;\n\telect.sync _|px, 0xffffffff;\n\tselp.u32 %0, 1, 0, px;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+__device__ __forceinline__ void umma_bf16_ss_warp(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                  uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, px;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "elect.sync _|px, 0xffffffff;\n\t"
+        "@px tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_bf16_ts_warp(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                  uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, px;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "elect.sync _|px, 0xffffffff;\n\t"
+        "@px tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_warp(uint64_t* bar) {
+    asm volatile(
+        "{\n\t.reg .pred px;\n\t"
+        "elect.sync _|px, 0xffffffff;\n\t"
+        "@px tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar))
         : "memory");
 }
 // Makes `bar` complete once every tcgen05.mma issued so far by this thread has finished.
