@@ -63,13 +63,14 @@ gdn_prefill_prep_kernel(const int32_t* __restrict__ cu, int num_seqs, int total_
 //   MMA1  [Q ; K] K^T            (128 x 64 x 128)  rows 0-63: Q K^T, rows 64-127: K K^T
 //   solve T = (I + A)^-1         fp32, one thread per ROW of T through the transposed system
 //                                y (I + A) = e_i  (backward substitution over columns)
-//   MMA2  [T''_a ; T''_b] K      (128 x 128 x 64)  T'' = T diag(beta o Gamma), bf16 hi + lo
+//   MMA2  [T''_a ; T''_b] K      (128 x 128 x 64)  T'' = T diag(beta o Gamma) in bf16
 constexpr int kIntraThreads = 128;
 constexpr uint32_t IQ_LO = 0, IK_LO = 8192, IQ_HI = 16384, IK_HI = 24576;  // TMA tiles [64][64] bf16
-constexpr uint32_t IT2 = 32768;      // T'' operand: hi [128][64] 16 KB | lo 16 KB
-constexpr uint32_t IAT = 65536;      // A^T for two heads, fp32 [2][64][kATP]
+constexpr uint32_t IT2 = 32768;      // T'' operand (bf16): [128][64] 16 KB
+constexpr uint32_t IAT = 49152;      // A^T for two heads, fp32 [2][64][kATP]
 constexpr int kATP = 68;
-constexpr uint32_t IGAM = IAT + 2 * 64 * kATP * 4;  // gam[2][64] | bet[2][64] | Gam[2][64] | tmp[4]
+constexpr uint32_t IYS = IAT + 2 * 64 * kATP * 4;   // columns 16..63 of the rows of T being solved, fp32 [48][128]
+constexpr uint32_t IGAM = IYS + 48 * 128 * 4;       // gam[2][64] | bet[2][64] | Gam[2][64] | tmp[4]
 constexpr uint32_t IBAR = IGAM + 6 * 64 * 4 + 64;
 constexpr uint32_t kIntraSmem = IBAR + 64 + 1024;
 constexpr uint32_t ITM_D1 = 0, ITM_D2 = 64, ITM_COLS = 256;
@@ -118,6 +119,12 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
     const uint32_t sb = smem_u32(smem);
     bool ok = true;
+#ifdef GDN_INTRA_PROFILE
+#define GDN_ISTAMP(slot) do { if (tid == 0) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)c * Hv + hq * G) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
+#else
+#define GDN_ISTAMP(slot) do { } while (0)
+#endif
+    GDN_ISTAMP(0);
 
     if (warp == 0) {
         if (elect_one()) {
@@ -131,6 +138,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         }
         __syncwarp();
         ok = mbar_wait_all(bar_load, 0, abort_flag);
+        GDN_ISTAMP(1);
         if (ok) {
             tc_fence_after_sync();
             constexpr uint32_t ID1 = umma_idesc_bf16(128, 64, false, false, false);
@@ -177,42 +185,44 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             if (!ok) break;
             tc_fence_after_sync();
         }
-        // ---- phase A: this thread's row of [Q K^T ; K K^T]: rows 0-63 -> P, rows 64-127 -> A^T
+        GDN_ISTAMP(2);
+        // ---- phase A: this thread's row of [Q K^T ; K K^T]: rows 0-63 -> P, rows 64-127 -> A^T.
+        // Sixteen columns at a time in a rolled loop: this kernel is long straight-line code and
+        // runs at instruction-fetch speed if its loops are fully unrolled.
         {
-            uint32_t r0[32], r1[32];
-            tmem_ld32(lane_addr + ITM_D1, r0);
-            tmem_ld32(lane_addr + ITM_D1 + 32, r1);
-            tmem_ld_wait();
             const int row = tid & 63;
-            for (int e = 0; e < nh; ++e) {
-                const float* gm = gam + e * 64;
-                const float gi = gm[row];
-                const int hv = hq * G + 2 * p + e;
-                if (tid < 64) {
-                    // P row: (Q K^T)_ij exp(gamma_i - gamma_j) for j <= i (difference masked before exp)
-                    uint8_t* wsP = ws + L.off_P + ((size_t)c * Hv + hv) * kPBytes;
+#pragma unroll 1
+            for (int q4 = 0; q4 < 4; ++q4) {
+                uint32_t r[16];
+                tmem_ld16(lane_addr + ITM_D1 + q4 * 16, r);
+                tmem_ld_wait();
+#pragma unroll 1
+                for (int e = 0; e < nh; ++e) {
+                    const float* gm = gam + e * 64 + q4 * 16;
+                    const float gi = gam[e * 64 + row];
+                    const int hv = hq * G + 2 * p + e;
+                    if (tid < 64) {
+                        // P row: (Q K^T)_ij exp(gamma_i - gamma_j) for j <= i (difference masked before exp)
+                        uint8_t* wsP = ws + L.off_P + ((size_t)c * Hv + hv) * kPBytes;
 #pragma unroll
-                    for (int c16 = 0; c16 < 8; ++c16) {
-                        uint32_t pk[4];
+                        for (int half = 0; half < 2; ++half) {
+                            uint32_t pk[4];
 #pragma unroll
-                        for (int q2 = 0; q2 < 4; ++q2) {
-                            const int j = c16 * 8 + q2 * 2;
-                            const float a0 = __uint_as_float(j < 32 ? r0[j] : r1[j - 32]);
-                            const float a1 = __uint_as_float(j + 1 < 32 ? r0[j + 1] : r1[j + 1 - 32]);
-                            const float p0 = (j <= row && row < len) ? a0 * __expf(gi - gm[j]) : 0.f;
-                            const float p1 = (j + 1 <= row && row < len) ? a1 * __expf(gi - gm[j + 1]) : 0.f;
-                            pk[q2] = pack_bf16x2(p0, p1);
+                            for (int q2 = 0; q2 < 4; ++q2) {
+                                const int jl = half * 8 + q2 * 2, j = q4 * 16 + jl;
+                                const float p0 = (j <= row && row < len) ? __uint_as_float(r[jl]) * __expf(gi - gm[jl]) : 0.f;
+                                const float p1 = (j + 1 <= row && row < len) ? __uint_as_float(r[jl + 1]) * __expf(gi - gm[jl + 1]) : 0.f;
+                                pk[q2] = pack_bf16x2(p0, p1);
+                            }
+                            *reinterpret_cast<uint4*>(wsP + swz(row, q4 * 2 + half)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         }
-                        *reinterpret_cast<uint4*>(wsP + swz(row, c16)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    }
-                } else {
-                    // A^T[j][i] = beta_i exp(gamma_i - gamma_j) (K K^T)_ij for j < i, else 0
-                    float* at = At + e * 64 * kATP;
-                    const float bi = bet[e * 64 + row];
+                    } else {
+                        // A^T[j][i] = beta_i exp(gamma_i - gamma_j) (K K^T)_ij for j < i, else 0
+                        float* at = At + e * 64 * kATP + (q4 * 16) * kATP + row;
+                        const float bi = bet[e * 64 + row];
 #pragma unroll
-                    for (int j = 0; j < 64; ++j) {
-                        const float a = __uint_as_float(j < 32 ? r0[j] : r1[j - 32]);
-                        at[j * kATP + row] = (j < row) ? bi * __expf(gi - gm[j]) * a : 0.f;
+                        for (int jl = 0; jl < 16; ++jl)
+                            at[jl * kATP] = (q4 * 16 + jl < row) ? bi * __expf(gi - gm[jl]) * __uint_as_float(r[jl]) : 0.f;
                     }
                 }
             }
@@ -225,77 +235,111 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             if (i == 0) wsS[128] = Gam[hh * 64 + len - 1];
         }
         __syncthreads();
-        // ---- UT transform, row i of T = (I + A)^-1:  y_j = delta_ij - sum_{m > j} y_m A[m][j]
-        float y[64];
-#pragma unroll
-        for (int j = 0; j < 64; ++j) y[j] = (j == i) ? 1.f : 0.f;
+        GDN_ISTAMP(3);
+        // ---- UT transform, row i of T = (I + A)^-1 through the transposed system
+        //      y_j = delta_ij - sum_{m > j} y_m A[m][j],
+        // in 16-column blocks from the right: the finished columns 16..63 of the row sit in this
+        // thread's private column of `ys`, the block being solved (and, at the end, columns 0..15)
+        // in registers.  Rows of the upper half of the chunk never reach the two right-hand blocks
+        // (y is zero there), so their warps skip them.
+        float yl[16];
         {
             const float* at = At + hh * 64 * kATP;
+            float* ys = reinterpret_cast<float*>(smem + IYS) + tid - 16 * 128;  // ys[m * 128] is column m >= 16
+            const int jb_top = (warp & 1) ? 3 : 1;  // highest 16-block with a nonzero entry for this warp's rows
+#pragma unroll 1
+            for (int jb = 3; jb > jb_top; --jb)
 #pragma unroll
-            for (int j = 62; j >= 0; --j) {
-                float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
-                const float* arow = at + j * kATP;
-                // m runs over (j, 63]; float4 groups that start above j
-                const int m0 = (j + 1 + 3) & ~3;
+                for (int jj = 0; jj < 16; ++jj) ys[(16 * jb + jj) * 128] = 0.f;
+#pragma unroll 1
+            for (int jb = jb_top; jb >= 0; --jb) {
+                float acc[16];
 #pragma unroll
-                for (int m = j + 1; m < m0 && m < 64; ++m) acc0 = fmaf(arow[m], y[m], acc0);
+                for (int jj = 0; jj < 16; ++jj) acc[jj] = 0.f;
+#pragma unroll 1
+                for (int m = 16 * jb_top + 12; m >= 16 * (jb + 1); m -= 4) {
+                    const float y0 = ys[(m + 0) * 128], y1 = ys[(m + 1) * 128], y2 = ys[(m + 2) * 128], y3 = ys[(m + 3) * 128];
 #pragma unroll
-                for (int m = m0; m < 64; m += 4) {
-                    const float4 a4 = *reinterpret_cast<const float4*>(arow + m);
-                    acc0 = fmaf(a4.x, y[m], acc0);
-                    acc1 = fmaf(a4.y, y[m + 1], acc1);
-                    acc2 = fmaf(a4.z, y[m + 2], acc2);
-                    acc3 = fmaf(a4.w, y[m + 3], acc3);
+                    for (int jj = 0; jj < 16; ++jj) {
+                        const float4 a4 = *reinterpret_cast<const float4*>(at + (16 * jb + jj) * kATP + m);
+                        acc[jj] = fmaf(a4.x, y0, fmaf(a4.y, y1, fmaf(a4.z, y2, fmaf(a4.w, y3, acc[jj]))));
+                    }
                 }
-                y[j] -= (acc0 + acc1) + (acc2 + acc3);
+#pragma unroll
+                for (int jj = 15; jj >= 0; --jj) {
+                    float sacc = acc[jj];
+                    const float* arow = at + (16 * jb + jj) * kATP + 16 * jb;
+#pragma unroll
+                    for (int mm = jj + 1; mm < 16; ++mm) sacc = fmaf(arow[mm], yl[mm], sacc);
+                    yl[jj] = ((16 * jb + jj) == i ? 1.f : 0.f) - sacc;
+                }
+                if (jb > 0) {
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj) ys[(16 * jb + jj) * 128] = yl[jj];
+                }
             }
         }
-        // ---- T' = T diag(beta) -> workspace (bf16 hi + lo); T'' = T' diag(Gamma) -> smem A operand (hi + lo)
+        GDN_ISTAMP(4);
+        // ---- T' = T diag(beta) -> workspace (bf16 hi + lo); T'' = T' diag(Gamma) -> smem A operand (bf16)
         {
             uint8_t* wsA = ws + L.off_A + ((size_t)c * Hv + h) * kABytes;
             const float* bt = bet + hh * 64;
             const float* Gm = Gam + hh * 64;
-#pragma unroll
-            for (int c16 = 0; c16 < 8; ++c16) {
-                uint32_t h1[4], l1[4], h2[4], l2[4];
+            const float* ys = reinterpret_cast<const float*>(smem + IYS) + tid - 16 * 128;
+            auto emit = [&](int c16, const float (&yv)[8]) {
+                uint32_t h1[4], l1[4], h2[4];
 #pragma unroll
                 for (int q2 = 0; q2 < 4; ++q2) {
                     const int j = c16 * 8 + q2 * 2;
-                    const float a0 = y[j] * bt[j], a1 = y[j + 1] * bt[j + 1];
+                    const float a0 = yv[q2 * 2] * bt[j], a1 = yv[q2 * 2 + 1] * bt[j + 1];
                     split_bf16x2(a0, a1, h1[q2], l1[q2]);
-                    split_bf16x2(a0 * Gm[j], a1 * Gm[j + 1], h2[q2], l2[q2]);
+                    h2[q2] = pack_bf16x2(a0 * Gm[j], a1 * Gm[j + 1]);
                 }
                 if (head_ok) {
                     *reinterpret_cast<uint4*>(wsA + swz(i, c16)) = make_uint4(h1[0], h1[1], h1[2], h1[3]);
                     *reinterpret_cast<uint4*>(wsA + 8192 + swz(i, c16)) = make_uint4(l1[0], l1[1], l1[2], l1[3]);
                 }
                 *reinterpret_cast<uint4*>(smem + IT2 + swz(tid, c16)) = make_uint4(h2[0], h2[1], h2[2], h2[3]);
-                *reinterpret_cast<uint4*>(smem + IT2 + 16384 + swz(tid, c16)) = make_uint4(l2[0], l2[1], l2[2], l2[3]);
+            };
+            {
+                const float ya[8] = {yl[0], yl[1], yl[2], yl[3], yl[4], yl[5], yl[6], yl[7]};
+                const float yb[8] = {yl[8], yl[9], yl[10], yl[11], yl[12], yl[13], yl[14], yl[15]};
+                emit(0, ya);
+                emit(1, yb);
+            }
+#pragma unroll 1
+            for (int c16 = 2; c16 < 8; ++c16) {
+                float yv[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) yv[e] = ys[(c16 * 8 + e) * 128];
+                emit(c16, yv);
             }
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncthreads();
+        GDN_ISTAMP(5);
         // ---- MMA2: W (both heads) = [T''_a ; T''_b] K, K read MN-major from the TMA tiles
         if (warp == 0) {
             tc_fence_after_sync();
             constexpr uint32_t ID2 = umma_idesc_bf16(128, 128, false, true, false);
-            const uint64_t dTh = umma_desc(sb + IT2, 16, 1024), dTl = umma_desc(sb + IT2 + 16384, 16, 1024);
+            const uint64_t dTh = umma_desc(sb + IT2, 16, 1024);
             const uint64_t dK = umma_desc(sb + IK_LO, IK_HI - IK_LO, 1024);
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) umma_bf16_ss_warp(tmem_base + ITM_D2, dTh + ks * 2, dK + ks * 128, ID2, ks > 0);
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks) umma_bf16_ss_warp(tmem_base + ITM_D2, dTl + ks * 2, dK + ks * 128, ID2, 1);
             umma_commit_warp(bar_mma2);
+            GDN_ISTAMP(8);
         }
         ok = mbar_wait_all(bar_mma2, (uint32_t)(p & 1), abort_flag);
+        GDN_ISTAMP(9);
         ok = __syncthreads_and(ok);
         if (!ok) break;
         tc_fence_after_sync();
+        GDN_ISTAMP(6);
         // ---- W row i of head h -> workspace (K-major B operand image: two [64][64] tiles)
         {
             uint8_t* wsW = ws + L.off_A + ((size_t)c * Hv + h) * kABytes + 16384;
-#pragma unroll
+#pragma unroll 1
             for (int b = 0; b < 4; ++b) {
                 uint32_t r[32];
                 tmem_ld32(lane_addr + ITM_D2 + b * 32, r);
@@ -314,6 +358,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
         }
         tc_fence_before_sync();
+        GDN_ISTAMP(7);
         __syncthreads();  // the next pair reuses A^T, the T'' tiles and the W accumulator
     }
 
