@@ -129,6 +129,39 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const flo
                           int Hqk, int Hv, int dk, int dv, void* stream);
 
 /*
+ * Prefill without a caller-provided workspace and without any allocation.  (The paper has no
+ * counterpart for this entry point; it exists for integration reasons only.)
+ *
+ * Who needs it: code that runs where device memory may not be allocated -- a plugin or
+ * operator called inside a framework whose memory pool is frozen for the duration of the call,
+ * a serving loop that pre-sized all of its buffers at start-up and forbids allocation on the
+ * request path, a host that has handed all of its device memory to another allocator.  Such
+ * callers can pass inputs and outputs they already own but have nowhere to get the
+ * gdn_prefill workspace from.
+ *
+ * Same arguments and results as gdn_prefill, minus the workspace.  The scratch is a fixed
+ * array of GDN_PREFILL_STATIC_SCRATCH_BYTES inside the library image: every device that
+ * loads the library holds those bytes until the process exits.  Problems whose workspace
+ * (gdn_prefill_workspace_bytes) exceeds that size are refused with GDN_ERR_WORKSPACE; nothing
+ * is launched in that case.  The call itself performs no cudaMalloc/cudaFree and calls no
+ * allocating library routine.
+ *
+ * The first call on each device looks up the array's device address (with that device
+ * current) and remembers it; make that first call outside any stream capture.
+ *
+ * All calls on a device share the one array, and it keeps whatever the previous call left in
+ * it.  Each call rewrites everything it later reads (the chunk table, the status word and
+ * every per-chunk block it uses), so stale contents are harmless, but two calls that overlap
+ * on the GPU -- different streams, or the same stream from two threads without ordering --
+ * race on the scratch and corrupt each other.  Serialise them.
+ */
+#define GDN_PREFILL_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+int gdn_prefill_static(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                       const int32_t* cu_seqlens, const float* initial_state, void* out, float* final_state,
+                       int total_tokens, int num_seqs, int max_seqlen,
+                       int Hqk, int Hv, int dk, int dv, void* stream);
+
+/*
  * Reads (and clears) the device-side status word that the prefill kernels set when a
  * bounded wait on an asynchronous copy or tensor-core completion ran out.  HOST
  * pointer out; synchronises `stream`.  *device_status == 0 means no kernel gave up.

@@ -19,7 +19,8 @@ STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL", 2: "GDN_ERR_SHAPE", 3: "GDN_ERR_
 
 # Every symbol include/gdn.h declares.
 EXPORTS = ("gdn_status_string", "gdn_decode", "gdn_decode_variant", "gdn_decode_num_variants",
-           "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_recurrent", "gdn_last_device_status")
+           "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_recurrent", "gdn_prefill_static",
+           "gdn_last_device_status")
 
 
 class GdnError(RuntimeError):
@@ -54,6 +55,8 @@ def lib() -> ctypes.CDLL:
         L.gdn_prefill.restype = I
         L.gdn_prefill_recurrent.argtypes = [P] * 9 + [I] * 7 + [P]
         L.gdn_prefill_recurrent.restype = I
+        L.gdn_prefill_static.argtypes = [P] * 9 + [I] * 7 + [P]
+        L.gdn_prefill_static.restype = I
         L.gdn_last_device_status.argtypes = [P, ctypes.POINTER(I), P]
         L.gdn_last_device_status.restype = I
         _lib = L
@@ -128,6 +131,25 @@ def gdn_prefill_recurrent(q, k, v, g, beta, cu_seqlens, initial_state, out, fina
                                      _ptr(initial_state), _ptr(out), _ptr(final_state), T, N, int(max_seqlen),
                                      Hqk, Hv, dk, dv, _stream(stream))
     _check(rc, "gdn_prefill_recurrent")
+
+
+PREFILL_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
+
+
+def gdn_prefill_static(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state, max_seqlen: int,
+                       stream=None) -> None:
+    """gdn_prefill for callers that cannot allocate device memory (a frozen memory pool, an
+    allocation-free request path): no workspace argument, the scratch is a fixed
+    PREFILL_STATIC_SCRATCH_BYTES array inside the library.  Raises GdnError(GDN_ERR_WORKSPACE)
+    when gdn_prefill_workspace_bytes(...) for the problem exceeds it.  Calls on one device must
+    not overlap on the GPU: they share that one array."""
+    T, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    N = cu_seqlens.shape[0] - 1
+    rc = lib().gdn_prefill_static(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(cu_seqlens),
+                                  _ptr(initial_state), _ptr(out), _ptr(final_state), T, N, int(max_seqlen),
+                                  Hqk, Hv, dk, dv, _stream(stream))
+    _check(rc, "gdn_prefill_static")
 
 
 def gdn_last_device_status(workspace, stream=None) -> int:
