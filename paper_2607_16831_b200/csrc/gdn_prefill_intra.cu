@@ -58,39 +58,48 @@ gdn_prefill_prep_kernel(const int32_t* __restrict__ cu, int num_seqs, int total_
 }
 
 // ------------------------------------------------------------------ intra-chunk kernel
-// One CTA (128 threads) per (chunk, q/k head); the G value heads that share the q/k head are
-// processed in pairs so that every tensor-core product has M = 128:
+// One CTA (128 threads, four CTAs per SM) per (chunk, q/k head, pair of value heads); a pair makes
+// every tensor-core product M = 128:
 //   MMA1  [Q ; K] K^T            (128 x 64 x 128)  rows 0-63: Q K^T, rows 64-127: K K^T
 //   solve T = (I + A)^-1         fp32, one thread per ROW of T through the transposed system
 //                                y (I + A) = e_i  (backward substitution over columns)
 //   MMA2  [T''_a ; T''_b] K      (128 x 128 x 64)  T'' = T diag(beta o Gamma) in bf16
+// The kernel is bound by the latency of the fp32 solve, so it is laid out for occupancy: 55 KB of
+// shared memory (the Q tiles are recycled for the rows being solved, A^T is kept as its ten
+// non-zero 16x16 blocks and later recycled for the T'' operand) and 128 tensor-memory columns.
 constexpr int kIntraThreads = 128;
 constexpr uint32_t IQ_LO = 0, IK_LO = 8192, IQ_HI = 16384, IK_HI = 24576;  // TMA tiles [64][64] bf16
-constexpr uint32_t IT2 = 32768;      // T'' operand (bf16): [128][64] 16 KB
-constexpr uint32_t IAT = 49152;      // A^T for two heads, fp32 [2][64][kATP]
-constexpr int kATP = 68;
-constexpr uint32_t IYS = IAT + 2 * 64 * kATP * 4;   // columns 16..63 of the rows of T being solved, fp32 [48][128]
-constexpr uint32_t IGAM = IYS + 48 * 128 * 4;       // gam[2][64] | bet[2][64] | Gam[2][64] | tmp[4]
+constexpr uint32_t IYS2 = IQ_LO, IYS3 = IQ_HI;  // after MMA1: columns 32-47 / 48-63 of the rows being solved, fp32 [16][128]
+constexpr uint32_t IAT = 32768;                 // A^T, two heads x ten 16x16 fp32 blocks (j-block <= m-block)
+constexpr uint32_t IT2 = IAT;                   // after the solve: T'' operand (bf16) [128][64]
+constexpr uint32_t IGAM = IAT + 2 * 10 * 1024;  // gam[2][64] | bet[2][64] | Gam[2][64] | tmp[4]
 constexpr uint32_t IBAR = IGAM + 6 * 64 * 4 + 64;
 constexpr uint32_t kIntraSmem = IBAR + 64 + 1024;
-constexpr uint32_t ITM_D1 = 0, ITM_D2 = 64, ITM_COLS = 256;
+constexpr uint32_t ITM_D1 = 0, ITM_D2 = 0, ITM_COLS = 128;  // the W accumulator reuses the columns of [QK^T ; KK^T]
 
-__global__ void __launch_bounds__(kIntraThreads)
+// index of the 16x16 block (j-block jb, m-block mb >= jb) of A^T
+__device__ __forceinline__ int at_blk(int jb, int mb) { return jb * 4 - (jb * (jb - 1)) / 2 + (mb - jb); }
+
+__global__ void __launch_bounds__(kIntraThreads, 4)
 gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const float* __restrict__ g, const float* __restrict__ beta, uint8_t* __restrict__ ws,
                          WsLayout L, int Hqk, int Hv) {
-    const int c = blockIdx.x, hq = blockIdx.y;
+    const int c = blockIdx.x;
     const int* hdr = reinterpret_cast<const int*>(ws);
     if (c >= hdr[1]) return;
+    const int G = Hv / Hqk;
+    const int npairs = (G + 1) / 2;
+    const int hq = blockIdx.y / npairs, p = blockIdx.y % npairs;
     const int4 info = reinterpret_cast<const int4*>(ws + L.off_chunk_info)[c];
     const int t0 = info.y, len = info.z;
-    const int G = Hv / Hqk;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int hh = tid >> 6, i = tid & 63;  // role in the gate / solve / W phases: head of the pair, row
+    const int nh = min(2, G - 2 * p);
+    const int h = hq * G + 2 * p + hh;      // this thread's value head in those phases
+    const bool head_ok = hh < nh;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    float* At = reinterpret_cast<float*>(smem + IAT);
     float* gam = reinterpret_cast<float*>(smem + IGAM);
     float* bet = gam + 128;
     float* Gam = gam + 256;
@@ -119,12 +128,6 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
     const uint32_t sb = smem_u32(smem);
     bool ok = true;
-#ifdef GDN_INTRA_PROFILE
-#define GDN_ISTAMP(slot) do { if (tid == 0) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)c * Hv + hq * G) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
-#else
-#define GDN_ISTAMP(slot) do { } while (0)
-#endif
-    GDN_ISTAMP(0);
 
     if (warp == 0) {
         if (elect_one()) {
@@ -137,8 +140,29 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tma_load_3d(smem + IK_HI, &map_k, bar_load, 64, hq, t0);
         }
         __syncwarp();
+    }
+    // ---- gates of both heads while the tiles are in flight: gamma = inclusive cumsum of g (fp32),
+    //      beta; both zero beyond len
+    {
+        float x = 0.f, b = 0.f;
+        if (head_ok && i < len) {
+            x = __ldg(g + (size_t)(t0 + i) * Hv + h);
+            b = __ldg(beta + (size_t)(t0 + i) * Hv + h);
+        }
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+        }
+        if ((warp & 1) == 0 && lane == 31) tmp[hh] = x;
+        __syncthreads();
+        if (warp & 1) x += tmp[hh];
+        gam[tid] = x;
+        bet[tid] = b;
+        Gam[tid] = __expf(x);
+    }
+    if (warp == 0) {
         ok = mbar_wait_all(bar_load, 0, abort_flag);
-        GDN_ISTAMP(1);
         if (ok) {
             tc_fence_after_sync();
             constexpr uint32_t ID1 = umma_idesc_bf16(128, 64, false, false, false);
@@ -149,48 +173,24 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) umma_bf16_ss_warp(tmem_base + ITM_D1, dA1 + ks * 2, dB1 + ks * 2, ID1, 1);
             umma_commit_warp(bar_mma1);
+            ok = mbar_wait_all(bar_mma1, 0, abort_flag);  // only this warp polls; the others park at the barrier
         }
     }
-
-    ok = __syncthreads_and(ok);  // uniform across the CTA: nobody enters the loop if the load gave up
-
-    const int npairs = (G + 1) / 2;
-    for (int p = 0; p < npairs && ok; ++p) {
-        const int nh = min(2, G - 2 * p);
-        const int h = hq * G + 2 * p + hh;  // this thread's value head in the gate / solve / W phases
-        const bool head_ok = hh < nh;
-        // ---- gates of both heads: gamma = inclusive cumsum of g (fp32), beta; zero beyond len
-        {
-            float x = 0.f, b = 0.f;
-            if (head_ok && i < len) {
-                x = __ldg(g + (size_t)(t0 + i) * Hv + h);
-                b = __ldg(beta + (size_t)(t0 + i) * Hv + h);
-            }
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const float y = __shfl_up_sync(0xffffffffu, x, o);
-                if (lane >= o) x += y;
-            }
-            if ((warp & 1) == 0 && lane == 31) tmp[hh] = x;
-            __syncthreads();
-            if (warp & 1) x += tmp[hh];
-            gam[tid] = x;
-            bet[tid] = b;
-            Gam[tid] = __expf(x);
-            __syncthreads();
+    ok = __syncthreads_and(ok);
+    if (ok) {
+        tc_fence_after_sync();
+        // per-token scalars of this thread's (head, row)
+        if (head_ok) {
+            float* wsS = reinterpret_cast<float*>(ws + L.off_scal + ((size_t)c * Hv + h) * kScalBytes);
+            wsS[i] = Gam[tid];
+            wsS[64 + i] = __expf(gam[hh * 64 + len - 1] - gam[tid]);
+            if (i == 0) wsS[128] = Gam[hh * 64 + len - 1];
         }
-        if (p == 0) {
-            ok = mbar_wait_all(bar_mma1, 0, abort_flag);
-            ok = __syncthreads_and(ok);
-            if (!ok) break;
-            tc_fence_after_sync();
-        }
-        GDN_ISTAMP(2);
-        // ---- phase A: this thread's row of [Q K^T ; K K^T]: rows 0-63 -> P, rows 64-127 -> A^T.
-        // Sixteen columns at a time in a rolled loop: this kernel is long straight-line code and
-        // runs at instruction-fetch speed if its loops are fully unrolled.
+        // ---- phase A: this thread's row of [Q K^T ; K K^T]: rows 0-63 -> P, rows 64-127 -> A^T,
+        //      sixteen columns at a time (rolled: long straight-line code runs at instruction-fetch speed)
         {
             const int row = tid & 63;
+            float* At = reinterpret_cast<float*>(smem + IAT);
 #pragma unroll 1
             for (int q4 = 0; q4 < 4; ++q4) {
                 uint32_t r[16];
@@ -200,10 +200,9 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 for (int e = 0; e < nh; ++e) {
                     const float* gm = gam + e * 64 + q4 * 16;
                     const float gi = gam[e * 64 + row];
-                    const int hv = hq * G + 2 * p + e;
                     if (tid < 64) {
                         // P row: (Q K^T)_ij exp(gamma_i - gamma_j) for j <= i (difference masked before exp)
-                        uint8_t* wsP = ws + L.off_P + ((size_t)c * Hv + hv) * kPBytes;
+                        uint8_t* wsP = ws + L.off_P + ((size_t)c * Hv + hq * G + 2 * p + e) * kPBytes;
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {
                             uint32_t pk[4];
@@ -216,76 +215,95 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                             }
                             *reinterpret_cast<uint4*>(wsP + swz(row, q4 * 2 + half)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         }
-                    } else {
-                        // A^T[j][i] = beta_i exp(gamma_i - gamma_j) (K K^T)_ij for j < i, else 0
-                        float* at = At + e * 64 * kATP + (q4 * 16) * kATP + row;
+                    } else if ((row >> 4) >= q4) {
+                        // A^T[j][i] = beta_i exp(gamma_i - gamma_j) (K K^T)_ij for j < i, else 0; block (q4, row/16)
+                        float* at = At + e * 10 * 256 + at_blk(q4, row >> 4) * 256 + (row & 15);
                         const float bi = bet[e * 64 + row];
 #pragma unroll
                         for (int jl = 0; jl < 16; ++jl)
-                            at[jl * kATP] = (q4 * 16 + jl < row) ? bi * __expf(gi - gm[jl]) * __uint_as_float(r[jl]) : 0.f;
+                            at[jl * 16] = (q4 * 16 + jl < row) ? bi * __expf(gi - gm[jl]) * __uint_as_float(r[jl]) : 0.f;
                     }
                 }
             }
         }
-        // per-token scalars of this thread's (head, row)
-        if (head_ok) {
-            float* wsS = reinterpret_cast<float*>(ws + L.off_scal + ((size_t)c * Hv + h) * kScalBytes);
-            wsS[i] = Gam[tid];
-            wsS[64 + i] = __expf(gam[hh * 64 + len - 1] - gam[tid]);
-            if (i == 0) wsS[128] = Gam[hh * 64 + len - 1];
-        }
-        __syncthreads();
-        GDN_ISTAMP(3);
+        tc_fence_before_sync();
+        __syncthreads();  // A^T complete; the Q tiles and the [QK^T ; KK^T] accumulator are dead from here on
+
         // ---- UT transform, row i of T = (I + A)^-1 through the transposed system
         //      y_j = delta_ij - sum_{m > j} y_m A[m][j],
-        // in 16-column blocks from the right: the finished columns 16..63 of the row sit in this
-        // thread's private column of `ys`, the block being solved (and, at the end, columns 0..15)
-        // in registers.  Rows of the upper half of the chunk never reach the two right-hand blocks
-        // (y is zero there), so their warps skip them.
-        float yl[16];
+        // in 16-column blocks from the right.  Finished columns 32..63 of the row sit in this thread's
+        // private column of ys2/ys3, columns 16..31 and the block being solved in registers.  Rows of
+        // the upper half of the chunk never reach the two right-hand blocks, so their warps skip them.
+        float yl[16], yl1[16];
+        const int top = (warp & 1) ? 3 : 1;  // highest 16-block with a nonzero entry for this warp's rows
         {
-            const float* at = At + hh * 64 * kATP;
-            float* ys = reinterpret_cast<float*>(smem + IYS) + tid - 16 * 128;  // ys[m * 128] is column m >= 16
-            const int jb_top = (warp & 1) ? 3 : 1;  // highest 16-block with a nonzero entry for this warp's rows
-#pragma unroll 1
-            for (int jb = 3; jb > jb_top; --jb)
+            const float* at = reinterpret_cast<const float*>(smem + IAT) + hh * 10 * 256;
+            float* ys2 = reinterpret_cast<float*>(smem + IYS2) + tid;
+            float* ys3 = reinterpret_cast<float*>(smem + IYS3) + tid;
 #pragma unroll
-                for (int jj = 0; jj < 16; ++jj) ys[(16 * jb + jj) * 128] = 0.f;
+            for (int jj = 0; jj < 16; ++jj) yl1[jj] = 0.f;
 #pragma unroll 1
-            for (int jb = jb_top; jb >= 0; --jb) {
+            for (int jb = top; jb >= 0; --jb) {
                 float acc[16];
 #pragma unroll
                 for (int jj = 0; jj < 16; ++jj) acc[jj] = 0.f;
+                // contributions of the finished blocks held in shared memory (m-blocks 3 and 2)
 #pragma unroll 1
-                for (int m = 16 * jb_top + 12; m >= 16 * (jb + 1); m -= 4) {
-                    const float y0 = ys[(m + 0) * 128], y1 = ys[(m + 1) * 128], y2 = ys[(m + 2) * 128], y3 = ys[(m + 3) * 128];
+                for (int mb = top; mb > jb && mb >= 2; --mb) {
+                    const float* blkp = at + at_blk(jb, mb) * 256;
+                    const float* yp = (mb == 3) ? ys3 : ys2;
+#pragma unroll 1
+                    for (int mg = 0; mg < 4; ++mg) {
+                        float4 a4[16];
 #pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) {
-                        const float4 a4 = *reinterpret_cast<const float4*>(at + (16 * jb + jj) * kATP + m);
-                        acc[jj] = fmaf(a4.x, y0, fmaf(a4.y, y1, fmaf(a4.z, y2, fmaf(a4.w, y3, acc[jj]))));
+                        for (int jj = 0; jj < 16; ++jj) a4[jj] = *reinterpret_cast<const float4*>(blkp + jj * 16 + mg * 4);
+                        const float y0 = yp[(mg * 4 + 0) * 128], y1 = yp[(mg * 4 + 1) * 128];
+                        const float y2 = yp[(mg * 4 + 2) * 128], y3 = yp[(mg * 4 + 3) * 128];
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj)
+                            acc[jj] = fmaf(a4[jj].x, y0, fmaf(a4[jj].y, y1, fmaf(a4[jj].z, y2, fmaf(a4[jj].w, y3, acc[jj]))));
                     }
                 }
+                // contribution of m-block 1 (in registers) to block 0
+                if (jb == 0) {
+                    const float* blkp = at + at_blk(0, 1) * 256;
 #pragma unroll
-                for (int jj = 15; jj >= 0; --jj) {
-                    float sacc = acc[jj];
-                    const float* arow = at + (16 * jb + jj) * kATP + 16 * jb;
+                    for (int mg = 0; mg < 4; ++mg) {
 #pragma unroll
-                    for (int mm = jj + 1; mm < 16; ++mm) sacc = fmaf(arow[mm], yl[mm], sacc);
-                    yl[jj] = ((16 * jb + jj) == i ? 1.f : 0.f) - sacc;
+                        for (int jj = 0; jj < 16; ++jj) {
+                            const float4 a4 = *reinterpret_cast<const float4*>(blkp + jj * 16 + mg * 4);
+                            acc[jj] = fmaf(a4.x, yl1[mg * 4], fmaf(a4.y, yl1[mg * 4 + 1],
+                                      fmaf(a4.z, yl1[mg * 4 + 2], fmaf(a4.w, yl1[mg * 4 + 3], acc[jj]))));
+                        }
+                    }
                 }
-                if (jb > 0) {
+                // diagonal 16x16 block, column by column from the right: once y_mm is known its
+                // contribution is pushed to every column left of it (independent FMAs, no long chain)
+                const float* ablk = at + at_blk(jb, jb) * 256;
 #pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) ys[(16 * jb + jj) * 128] = yl[jj];
+                for (int mm = 15; mm >= 0; --mm) {
+                    yl[mm] = ((16 * jb + mm) == i ? 1.f : 0.f) - acc[mm];
+#pragma unroll
+                    for (int jj = 0; jj < mm; ++jj) acc[jj] = fmaf(ablk[jj * 16 + mm], yl[mm], acc[jj]);
+                }
+                if (jb == 3) {
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj) ys3[jj * 128] = yl[jj];
+                } else if (jb == 2) {
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj) ys2[jj * 128] = yl[jj];
+                } else if (jb == 1) {
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj) yl1[jj] = yl[jj];
                 }
             }
         }
-        GDN_ISTAMP(4);
+        __syncthreads();  // every warp is done with A^T: its space becomes the T'' operand
         // ---- T' = T diag(beta) -> workspace (bf16 hi + lo); T'' = T' diag(Gamma) -> smem A operand (bf16)
         {
             uint8_t* wsA = ws + L.off_A + ((size_t)c * Hv + h) * kABytes;
             const float* bt = bet + hh * 64;
             const float* Gm = Gam + hh * 64;
-            const float* ys = reinterpret_cast<const float*>(smem + IYS) + tid - 16 * 128;
             auto emit = [&](int c16, const float (&yv)[8]) {
                 uint32_t h1[4], l1[4], h2[4];
 #pragma unroll
@@ -302,23 +320,27 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 *reinterpret_cast<uint4*>(smem + IT2 + swz(tid, c16)) = make_uint4(h2[0], h2[1], h2[2], h2[3]);
             };
             {
-                const float ya[8] = {yl[0], yl[1], yl[2], yl[3], yl[4], yl[5], yl[6], yl[7]};
-                const float yb[8] = {yl[8], yl[9], yl[10], yl[11], yl[12], yl[13], yl[14], yl[15]};
-                emit(0, ya);
-                emit(1, yb);
+                const float a[8] = {yl[0], yl[1], yl[2], yl[3], yl[4], yl[5], yl[6], yl[7]};
+                const float b[8] = {yl[8], yl[9], yl[10], yl[11], yl[12], yl[13], yl[14], yl[15]};
+                const float cc[8] = {yl1[0], yl1[1], yl1[2], yl1[3], yl1[4], yl1[5], yl1[6], yl1[7]};
+                const float d[8] = {yl1[8], yl1[9], yl1[10], yl1[11], yl1[12], yl1[13], yl1[14], yl1[15]};
+                emit(0, a);
+                emit(1, b);
+                emit(2, cc);
+                emit(3, d);
             }
 #pragma unroll 1
-            for (int c16 = 2; c16 < 8; ++c16) {
+            for (int c16 = 4; c16 < 8; ++c16) {
+                const float* yp = reinterpret_cast<const float*>(smem + (c16 < 6 ? IYS2 : IYS3)) + tid + ((c16 & 1) * 8) * 128;
                 float yv[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) yv[e] = ys[(c16 * 8 + e) * 128];
+                for (int e = 0; e < 8; ++e) yv[e] = (top == 3) ? yp[e * 128] : 0.f;
                 emit(c16, yv);
             }
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncthreads();
-        GDN_ISTAMP(5);
         // ---- MMA2: W (both heads) = [T''_a ; T''_b] K, K read MN-major from the TMA tiles
         if (warp == 0) {
             tc_fence_after_sync();
@@ -328,38 +350,31 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) umma_bf16_ss_warp(tmem_base + ITM_D2, dTh + ks * 2, dK + ks * 128, ID2, ks > 0);
             umma_commit_warp(bar_mma2);
-            GDN_ISTAMP(8);
+            ok = mbar_wait_all(bar_mma2, 0, abort_flag);
         }
-        ok = mbar_wait_all(bar_mma2, (uint32_t)(p & 1), abort_flag);
-        GDN_ISTAMP(9);
         ok = __syncthreads_and(ok);
-        if (!ok) break;
+    }
+    if (ok) {
         tc_fence_after_sync();
-        GDN_ISTAMP(6);
         // ---- W row i of head h -> workspace (K-major B operand image: two [64][64] tiles)
-        {
-            uint8_t* wsW = ws + L.off_A + ((size_t)c * Hv + h) * kABytes + 16384;
+        uint8_t* wsW = ws + L.off_A + ((size_t)c * Hv + h) * kABytes + 16384;
 #pragma unroll 1
-            for (int b = 0; b < 4; ++b) {
-                uint32_t r[32];
-                tmem_ld32(lane_addr + ITM_D2 + b * 32, r);
-                tmem_ld_wait();
-                if (head_ok) {
+        for (int b = 0; b < 4; ++b) {
+            uint32_t r[32];
+            tmem_ld32(lane_addr + ITM_D2 + b * 32, r);
+            tmem_ld_wait();
+            if (head_ok) {
 #pragma unroll
-                    for (int cc = 0; cc < 4; ++cc) {
-                        uint4 o;
-                        o.x = pack_bf16x2(__uint_as_float(r[cc * 8 + 0]), __uint_as_float(r[cc * 8 + 1]));
-                        o.y = pack_bf16x2(__uint_as_float(r[cc * 8 + 2]), __uint_as_float(r[cc * 8 + 3]));
-                        o.z = pack_bf16x2(__uint_as_float(r[cc * 8 + 4]), __uint_as_float(r[cc * 8 + 5]));
-                        o.w = pack_bf16x2(__uint_as_float(r[cc * 8 + 6]), __uint_as_float(r[cc * 8 + 7]));
-                        *reinterpret_cast<uint4*>(wsW + (b >> 1) * 8192 + swz(i, (b & 1) * 4 + cc)) = o;
-                    }
+                for (int cc = 0; cc < 4; ++cc) {
+                    uint4 o;
+                    o.x = pack_bf16x2(__uint_as_float(r[cc * 8 + 0]), __uint_as_float(r[cc * 8 + 1]));
+                    o.y = pack_bf16x2(__uint_as_float(r[cc * 8 + 2]), __uint_as_float(r[cc * 8 + 3]));
+                    o.z = pack_bf16x2(__uint_as_float(r[cc * 8 + 4]), __uint_as_float(r[cc * 8 + 5]));
+                    o.w = pack_bf16x2(__uint_as_float(r[cc * 8 + 6]), __uint_as_float(r[cc * 8 + 7]));
+                    *reinterpret_cast<uint4*>(wsW + (b >> 1) * 8192 + swz(i, (b & 1) * 4 + cc)) = o;
                 }
             }
         }
-        tc_fence_before_sync();
-        GDN_ISTAMP(7);
-        __syncthreads();  // the next pair reuses A^T, the T'' tiles and the W accumulator
     }
 
     if (*abort_flag && tid == 0) atomicExch(reinterpret_cast<int*>(ws), kStatusTimeout);
@@ -388,7 +403,8 @@ cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, c
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    dim3 grid(L.nc_max, Hqk);
+    const int G = Hv / Hqk;
+    dim3 grid(L.nc_max, Hqk * ((G + 1) / 2));
     gdn_prefill_intra_kernel<<<grid, kIntraThreads, kIntraSmem, st>>>(mq, mk, g, beta, ws, L, Hqk, Hv);
     return cudaGetLastError();
 }
