@@ -119,9 +119,13 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
     if (warp == 8) {
         // =========================================================== issuer: MMA
-        // The whole warp runs this loop in lock step; one elected lane issues each MMA.
+        // The whole warp runs this loop in lock step; one elected lane issues each MMA.  Values that
+        // feed the MMA operands are broadcast from lane 0 so that the compiler knows they are
+        // warp-uniform and keeps descriptors and addresses in uniform registers.
         {
-            const uint32_t sb = smem_u32(smem);
+            const uint32_t sb = __shfl_sync(0xffffffffu, smem_u32(smem), 0);
+            const uint32_t tmem_base_u = __shfl_sync(0xffffffffu, tmem_base, 0);
+            const int nchunks_u = __shfl_sync(0xffffffffu, nchunks, 0);
             constexpr uint32_t ID_G1 = umma_idesc_bf16(128, 64, true, false, false);    // V^T (MN-major A) x T'^T
             constexpr uint32_t ID_G2A = umma_idesc_bf16(128, 64, false, false, true);   // -(S) x W^T
             constexpr uint32_t ID_N64 = umma_idesc_bf16(128, 64, false, false, false);  // S x Q^T ; Delta^T x P^T
@@ -139,22 +143,22 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 const uint64_t so = st * kStageStep;
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
-                    umma_bf16_ss_warp(tmem_base + TM_DELTA, dV + so + ks * 128, dThi + so + ks * 2, ID_G1, ks > 0);
+                    umma_bf16_ss_warp(tmem_base_u + TM_DELTA, dV + so + ks * 128, dThi + so + ks * 2, ID_G1, ks > 0);
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
-                    umma_bf16_ss_warp(tmem_base + TM_DELTA, dV + so + ks * 128, dTlo + so + ks * 2, ID_G1, 1);
+                    umma_bf16_ss_warp(tmem_base_u + TM_DELTA, dV + so + ks * 128, dTlo + so + ks * 2, ID_G1, 1);
             };
 
             bool g1_issued = false;
 
 #define GDN_WAIT(idx, parity) if (!mbar_wait_all(bars + (idx), (uint32_t)(parity), abort_flag)) break
 
-            for (int ci = 0; ci < nchunks; ++ci) {
+            for (int ci = 0; ci < nchunks_u; ++ci) {
                 const int c = c_begin + ci;
                 (void)c;
                 const int st = ci & 1, par = ci & 1, ph2 = (ci >> 1) & 1;
                 const uint64_t so = st * kStageStep;
-                const bool last = (ci + 1 == nchunks);
+                const bool last = (ci + 1 == nchunks_u);
                 if (lane == 0) GDN_STAMP(c, 0);
                 if (!g1_issued) {
                     GDN_WAIT(B_FULL_A0 + st, ph2);
@@ -166,18 +170,26 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 GDN_WAIT(B_SHI, par);
                 if (lane == 0) GDN_STAMP(c, 2);
                 tc_fence_after_sync();
+                {
+                    const uint64_t w0 = dW0 + so, w1 = dW1 + so;
+                    const uint32_t td = tmem_base_u + TM_DELTA, ta = tmem_base_u + TM_SHI;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    umma_bf16_ts_warp(tmem_base + TM_DELTA, tmem_base + TM_SHI + ks * 8,
-                                 (ks < 4 ? dW0 : dW1) + so + (ks & 3) * 2, ID_G2A, 1);
+                    for (int ks = 0; ks < 4; ++ks) umma_bf16_ts_warp(td, ta + ks * 8, w0 + ks * 2, ID_G2A, 1);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) umma_bf16_ts_warp(td, ta + 32 + ks * 8, w1 + ks * 2, ID_G2A, 1);
+                }
                 umma_commit_warp(bars + B_DELTA);
                 if (lane == 0) GDN_STAMP(c, 4);
                 // ---- off the chain: Oa^T = S Q^T (runs while the chain warps drain Delta^T)
                 if (ci >= 1) GDN_WAIT(B_OFREE, par ^ 1);
+                {
+                    const uint64_t q0 = dQ0 + so, q1 = dQ1 + so;
+                    const uint32_t td = tmem_base_u + TM_OA, ta = tmem_base_u + TM_SHI;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)
-                    umma_bf16_ts_warp(tmem_base + TM_OA, tmem_base + TM_SHI + ks * 8,
-                                 (ks < 4 ? dQ0 : dQ1) + so + (ks & 3) * 2, ID_N64, ks > 0);
+                    for (int ks = 0; ks < 4; ++ks) umma_bf16_ts_warp(td, ta + ks * 8, q0 + ks * 2, ID_N64, ks > 0);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) umma_bf16_ts_warp(td, ta + 32 + ks * 8, q1 + ks * 2, ID_N64, 1);
+                }
                 if (lane == 0) GDN_STAMP(c, 5);
                 // ---- on the chain: S += (e o Delta)^T K  (hi + lo; A in tensor memory, B = K MN-major)
                 GDN_WAIT(B_FULL_B0 + st, ph2);
@@ -186,19 +198,22 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 GDN_WAIT(B_DW, par);
                 if (lane == 0) GDN_STAMP(c, 8);
                 tc_fence_after_sync();
+                {
+                    const uint64_t k0 = dK + so;
+                    const uint32_t td = tmem_base_u + TM_S;
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_bf16_ts_warp(tmem_base + TM_S, tmem_base + TM_DTH + ks * 8, dK + so + ks * 128, ID_G3B, 1);
+                    for (int ks = 0; ks < 4; ++ks) umma_bf16_ts_warp(td, tmem_base_u + TM_DTH + ks * 8, k0 + ks * 128, ID_G3B, 1);
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_bf16_ts_warp(tmem_base + TM_S, tmem_base + TM_DTL + ks * 8, dK + so + ks * 128, ID_G3B, 1);
+                    for (int ks = 0; ks < 4; ++ks) umma_bf16_ts_warp(td, tmem_base_u + TM_DTL + ks * 8, k0 + ks * 128, ID_G3B, 1);
+                }
                 umma_commit_warp(bars + B_STATE);
                 if (lane == 0) GDN_STAMP(c, 9);
                 // ---- off the chain: Ob^T = Delta^T P^T, and the next chunk's V^T T'^T if it has landed
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
-                    umma_bf16_ts_warp(tmem_base + TM_OB, tmem_base + TM_DL + ks * 8, dP + so + ks * 2, ID_N64, ks > 0);
-                if (!last && __shfl_sync(0xffffffffu, lane == 0 ? (uint32_t)mbar_try_wait(bars + B_FULL_A0 + (st ^ 1), ((ci + 1) >> 1) & 1) : 0u, 0)) {
+                    umma_bf16_ts_warp(tmem_base_u + TM_OB, tmem_base_u + TM_DL + ks * 8, dP + so + ks * 2, ID_N64, ks > 0);
+                if (!last) {
+                    GDN_WAIT(B_FULL_A0 + (st ^ 1), ((ci + 1) >> 1) & 1);  // requested a whole chunk ago
                     tc_fence_after_sync();
                     issue_G1(st ^ 1);
                     g1_issued = true;
@@ -398,26 +413,31 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             if (!mbar_wait_all(bars + B_O, par, abort_flag)) break;
             tc_fence_after_sync();
             if (tid == 128) GDN_STAMP(c, 25);
-            // o_i = Gamma_i Oa^T[v][i] + Ob^T[v][i], packed two tokens per register
-            uint32_t op[32];
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t a[32], b[32];
-                tmem_ld32(lane_addr + TM_OA + half * 32, a);
-                tmem_ld32(lane_addr + TM_OB + half * 32, b);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j4 = 0; j4 < 8; ++j4) {
-                    const float4 gm = __ldg(g4 + half * 8 + j4);
-                    op[half * 16 + j4 * 2] = pack_bf16x2(fmaf(gm.x, __uint_as_float(a[4 * j4]), __uint_as_float(b[4 * j4])),
-                                                         fmaf(gm.y, __uint_as_float(a[4 * j4 + 1]), __uint_as_float(b[4 * j4 + 1])));
-                    op[half * 16 + j4 * 2 + 1] = pack_bf16x2(fmaf(gm.z, __uint_as_float(a[4 * j4 + 2]), __uint_as_float(b[4 * j4 + 2])),
-                                                             fmaf(gm.w, __uint_as_float(a[4 * j4 + 3]), __uint_as_float(b[4 * j4 + 3])));
-                }
-            }
+            // drain both accumulators into registers and hand the columns back at once: the next
+            // chunk's S Q^T is waiting for them
+            uint32_t a0[32], a1[32], b0[32], b1[32];
+            tmem_ld32(lane_addr + TM_OA, a0);
+            tmem_ld32(lane_addr + TM_OA + 32, a1);
+            tmem_ld32(lane_addr + TM_OB, b0);
+            tmem_ld32(lane_addr + TM_OB + 32, b1);
+            tmem_ld_wait();
             tc_fence_before_sync();
             mbar_arrive(bars + B_OFREE);
             if (tid == 128) GDN_STAMP(c, 26);
+            // o_i = Gamma_i Oa^T[v][i] + Ob^T[v][i], packed two tokens per register
+            uint32_t op[32];
+#pragma unroll
+            for (int j4 = 0; j4 < 8; ++j4) {
+                const float4 gm = __ldg(g4 + j4), gn = __ldg(g4 + 8 + j4);
+                op[j4 * 2] = pack_bf16x2(fmaf(gm.x, __uint_as_float(a0[4 * j4]), __uint_as_float(b0[4 * j4])),
+                                         fmaf(gm.y, __uint_as_float(a0[4 * j4 + 1]), __uint_as_float(b0[4 * j4 + 1])));
+                op[j4 * 2 + 1] = pack_bf16x2(fmaf(gm.z, __uint_as_float(a0[4 * j4 + 2]), __uint_as_float(b0[4 * j4 + 2])),
+                                             fmaf(gm.w, __uint_as_float(a0[4 * j4 + 3]), __uint_as_float(b0[4 * j4 + 3])));
+                op[16 + j4 * 2] = pack_bf16x2(fmaf(gn.x, __uint_as_float(a1[4 * j4]), __uint_as_float(b1[4 * j4])),
+                                              fmaf(gn.y, __uint_as_float(a1[4 * j4 + 1]), __uint_as_float(b1[4 * j4 + 1])));
+                op[16 + j4 * 2 + 1] = pack_bf16x2(fmaf(gn.z, __uint_as_float(a1[4 * j4 + 2]), __uint_as_float(b1[4 * j4 + 2])),
+                                                  fmaf(gn.w, __uint_as_float(a1[4 * j4 + 3]), __uint_as_float(b1[4 * j4 + 3])));
+            }
             uint16_t* orow = out + ((size_t)t0 * Hv + h) * kD + v;
             const size_t ostride = (size_t)Hv * kD;
 #pragma unroll
