@@ -60,7 +60,8 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                          const __grid_constant__ CUtensorMap map_v, const float* initial_state,
                          uint16_t* __restrict__ out, float* final_state, uint8_t* __restrict__ ws, WsLayout L,
                          int Hqk, int Hv) {
-    const int h = blockIdx.x % Hv, n = blockIdx.x / Hv;
+    // CTAs are handed out longest sequence first
+    const int h = blockIdx.x % Hv, n = reinterpret_cast<const int*>(ws + L.off_seq_order)[blockIdx.x / Hv];
     const int hq = h / (Hv / Hqk);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 

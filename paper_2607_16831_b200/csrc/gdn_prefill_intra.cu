@@ -19,7 +19,7 @@ using namespace sm100;
 // ------------------------------------------------------------------ prep: chunk table
 __global__ void __launch_bounds__(256)
 gdn_prefill_prep_kernel(const int32_t* __restrict__ cu, int num_seqs, int total_tokens, int* hdr,
-                        int* chunk_off, int4* chunk_info, int nc_max) {
+                        int* chunk_off, int* seq_order, int4* chunk_info, int nc_max) {
     __shared__ int part[257];
     const int tid = threadIdx.x;
     const int per = (num_seqs + 255) / 256;
@@ -54,6 +54,18 @@ gdn_prefill_prep_kernel(const int32_t* __restrict__ cu, int num_seqs, int total_
         for (int j = 0; j < nch; ++j)
             if (base + j < nc_max) chunk_info[base + j] = make_int4(n, t0 + j * kChunk, min(kChunk, t1 - t0 - j * kChunk), j);
         base += nch;
+    }
+    // Longest sequences first: the chain kernel runs one CTA per (sequence, head) and its cost is
+    // the chunk count, so handing out the long chains first shortens the tail of the launch.
+    // Rank by counting (ties broken by index); O(N^2 / 256) per thread is fine for any sane batch.
+    for (int n = tid; n < num_seqs; n += 256) {
+        const int ln = max(0, min(cu[n + 1], total_tokens)) - max(0, min(cu[n], total_tokens));
+        int rank = 0;
+        for (int m = 0; m < num_seqs; ++m) {
+            const int lm = max(0, min(cu[m + 1], total_tokens)) - max(0, min(cu[m], total_tokens));
+            rank += (lm > ln) || (lm == ln && m < n);
+        }
+        seq_order[rank] = n;
     }
 }
 
@@ -390,6 +402,7 @@ cudaError_t launch_prefill_prep(const int32_t* cu_seqlens, int num_seqs, int tot
                                 const WsLayout& L, cudaStream_t st) {
     gdn_prefill_prep_kernel<<<1, 256, 0, st>>>(cu_seqlens, num_seqs, total_tokens, reinterpret_cast<int*>(ws),
                                                reinterpret_cast<int*>(ws + L.off_chunk_off),
+                                               reinterpret_cast<int*>(ws + L.off_seq_order),
                                                reinterpret_cast<int4*>(ws + L.off_chunk_info), L.nc_max);
     return cudaGetLastError();
 }

@@ -15,7 +15,7 @@ constexpr int kStatusTimeout = 1;  // device status: a bounded wait ran out
 
 struct WsLayout {
     int nc_max;
-    size_t off_chunk_off, off_chunk_info, off_scal, off_A, off_P, total;
+    size_t off_chunk_off, off_seq_order, off_chunk_info, off_scal, off_A, off_P, total;
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -26,6 +26,8 @@ __host__ __device__ inline WsLayout ws_layout(int total_tokens, int num_seqs, in
     size_t o = 1024;                              // header: [0] status, [1] total chunks
     L.off_chunk_off = o;
     o = align_up(o + sizeof(int) * (size_t)(num_seqs + 1), 1024);
+    L.off_seq_order = o;                          // sequences by decreasing chunk count
+    o = align_up(o + sizeof(int) * (size_t)num_seqs, 1024);
     L.off_chunk_info = o;
     o = align_up(o + sizeof(int4) * (size_t)L.nc_max, 1024);
     L.off_scal = o;

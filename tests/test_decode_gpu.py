@@ -73,3 +73,42 @@ def test_decode_empty_batch_is_ok():
     eg = torch.empty((0, 32), dtype=torch.float32, device="cuda")
     es = torch.empty((0, 32, 128, 128), dtype=torch.float32, device="cuda")
     gdn.gdn_decode(e, e, ev, eg, eg, es, es, ev)
+
+
+def test_decode_guard_bands_stay_intact():
+    import torch
+    import paper_2607_16831_b200 as gdn
+    cfg = config("decode_sweep", B=3, seed=21)
+    tok = cfg["tokens"]
+    d = harness.to_device(tok)
+    s_in = torch.from_numpy(cfg["state"]).cuda()
+    so_buf = torch.full((5, 32, 128, 128), 7.0, dtype=torch.float32, device="cuda")
+    o_buf = torch.full((5, 32, 128), 7.0, dtype=torch.bfloat16, device="cuda")
+    gdn.gdn_decode(d["q"], d["k"], d["v"], d["g"], d["beta"], s_in, so_buf[1:4], o_buf[1:4])
+    torch.cuda.synchronize()
+    assert torch.all(so_buf[0] == 7.0) and torch.all(so_buf[4] == 7.0)
+    assert torch.all(o_buf[0] == 7.0) and torch.all(o_buf[4] == 7.0)
+    ref_o, ref_s = oracle.decode(*harness.token_arrays(tok), cfg["state"])
+    harness.assert_close(harness.bf16_to_numpy(o_buf[1:4]), ref_o, so_buf[1:4].cpu().numpy().astype(np.float64), ref_s, "decode guard")
+
+
+def test_decode_then_prefill_state_handoff():
+    """T decode calls from a state == one prefill of the same T tokens from that state."""
+    import torch
+    import paper_2607_16831_b200 as gdn
+    from gdn_inputs import make_cu_seqlens, make_state, make_tokens
+    T, Hqk, Hv = 9, 2, 4
+    tok = make_tokens(T, Hqk, Hv, seed=25, gate_mean=4.0)
+    init = make_state(1, Hv, seed=25)
+    pre = harness.run_prefill(dict(tokens=tok, cu_seqlens=make_cu_seqlens([T]), initial_state=init))
+    d = harness.to_device(tok)
+    s = torch.from_numpy(init).cuda()
+    outs = []
+    for t in range(T):
+        o = torch.empty((1, Hv, 128), dtype=torch.bfloat16, device="cuda")
+        gdn.gdn_decode(d["q"][t:t + 1], d["k"][t:t + 1], d["v"][t:t + 1], d["g"][t:t + 1], d["beta"][t:t + 1], s, s, o)
+        outs.append(harness.bf16_to_numpy(o))
+    torch.cuda.synchronize()
+    dec_out = np.concatenate(outs, axis=0)
+    assert harness.rel_fro(dec_out, pre["out"]) < 8e-3
+    assert harness.rel_fro(s.cpu().numpy().astype(np.float64), pre["final_state"]) < 5e-3

@@ -93,3 +93,75 @@ def test_prefill_long_weak_decay():
 
 def test_prefill_varlen_config():
     check(config("prefill_varlen"), "prefill varlen 16 x U[1,2048]")
+
+
+@pytest.mark.parametrize("Hqk,Hv", [(2, 2), (1, 4), (1, 3), (3, 6)])
+def test_prefill_head_groupings(Hqk, Hv):
+    """G = Hv/Hqk of 1, 4, 3 (odd: the last pair of value heads is half empty) and 2."""
+    check(custom([90, 130], Hqk, Hv, seed=23 + Hv), "prefill heads %d/%d" % (Hqk, Hv))
+
+
+def test_prefill_correlated_keys_stress():
+    """Keys sharing a common direction make the intra-chunk triangular system far from the identity."""
+    e = check(custom([256], 2, 4, seed=29, gate_mean=6.0, key_correlation=0.5), "prefill correlated keys")
+    assert e["state_rel_fro"] < 4e-3
+
+
+def test_prefill_final_state_may_alias_initial_state_and_guard_bands_stay_intact():
+    import torch
+    import paper_2607_16831_b200 as gdn
+
+    cfg = custom([70, 33], 2, 4, seed=31)
+    tok = cfg["tokens"]
+    d = harness.to_device(tok)
+    cu_np = np.asarray(cfg["cu_seqlens"], dtype=np.int32)
+    cu = torch.from_numpy(cu_np).cuda()
+    T, N, Hv = tok.T, 2, 4
+    pad = 64  # canary rows around the outputs
+    out_buf = torch.full((T + 2 * pad, Hv, 128), 7.0, dtype=torch.bfloat16, device="cuda")
+    st_buf = torch.full((N + 2, Hv, 128, 128), 7.0, dtype=torch.float32, device="cuda")
+    st_buf[1:N + 1] = torch.from_numpy(cfg["initial_state"]).cuda()
+    out, state = out_buf[pad:pad + T], st_buf[1:N + 1]
+    ws = harness.alloc_workspace(T, N, tok.Hqk, Hv)
+    gdn.gdn_prefill(d["q"], d["k"], d["v"], d["g"], d["beta"], cu, state, out, state, int(np.max(np.diff(cu_np))), ws)
+    torch.cuda.synchronize()
+    assert gdn.gdn_last_device_status(ws) == 0
+    ref_o, ref_s = oracle.prefill(*harness.token_arrays(tok), cfg["cu_seqlens"], cfg["initial_state"])
+    harness.assert_close(harness.bf16_to_numpy(out), ref_o, state.cpu().numpy().astype(np.float64), ref_s, "in-place state")
+    assert torch.all(out_buf[:pad] == 7.0) and torch.all(out_buf[pad + T:] == 7.0), "wrote outside `out`"
+    assert torch.all(st_buf[0] == 7.0) and torch.all(st_buf[N + 1] == 7.0), "wrote outside `final_state`"
+
+
+def test_prefill_workspace_errors_are_reported_before_any_launch():
+    import torch
+    import paper_2607_16831_b200 as gdn
+
+    cfg = custom([64], 1, 1, seed=37)
+    tok = cfg["tokens"]
+    d = harness.to_device(tok)
+    cu = torch.from_numpy(np.asarray(cfg["cu_seqlens"], dtype=np.int32)).cuda()
+    out = torch.empty((64, 1, 128), dtype=torch.bfloat16, device="cuda")
+    ws = harness.alloc_workspace(64, 1, 1, 1)
+    for bad in (None, ws[: ws.numel() // 2], ws[16:]):  # missing, too small, misaligned
+        with pytest.raises(gdn.GdnError) as err:
+            gdn.gdn_prefill(d["q"], d["k"], d["v"], d["g"], d["beta"], cu, None, out, None, 64, bad)
+        assert err.value.status == 4
+
+
+def test_prefill_malformed_cu_seqlens_stays_in_bounds():
+    """Offsets beyond total_tokens are clamped on the device: results are unspecified but no
+    access leaves the buffers (the canaries survive and the call completes)."""
+    import torch
+    import paper_2607_16831_b200 as gdn
+
+    tok = make_tokens(100, 1, 2, seed=41)
+    d = harness.to_device(tok)
+    cu = torch.tensor([0, 60, 500], dtype=torch.int32, device="cuda")  # claims 500 tokens, only 100 exist
+    out_buf = torch.full((100 + 128, 2, 128), 7.0, dtype=torch.bfloat16, device="cuda")
+    fin = torch.empty((2, 2, 128, 128), dtype=torch.float32, device="cuda")
+    ws = harness.alloc_workspace(100, 2, 1, 2)
+    gdn.gdn_prefill(d["q"], d["k"], d["v"], d["g"], d["beta"], cu, None, out_buf[:100], fin, 100, ws)
+    torch.cuda.synchronize()
+    assert gdn.gdn_last_device_status(ws) == 0
+    assert torch.all(out_buf[100:] == 7.0)
+    assert torch.isfinite(fin).all()
