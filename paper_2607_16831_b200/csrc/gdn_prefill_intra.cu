@@ -71,26 +71,33 @@ gdn_prefill_prep_kernel(const int32_t* __restrict__ cu, int num_seqs, int total_
 
 // ------------------------------------------------------------------ intra-chunk kernel
 // One CTA (128 threads, four CTAs per SM) per (chunk, q/k head, pair of value heads); a pair makes
-// every tensor-core product M = 128:
-//   MMA1  [Q ; K] K^T            (128 x 64 x 128)  rows 0-63: Q K^T, rows 64-127: K K^T
-//   solve T = (I + A)^-1         fp32, one thread per ROW of T through the transposed system
-//                                y (I + A) = e_i  (backward substitution over columns)
-//   MMA2  [T''_a ; T''_b] K      (128 x 128 x 64)  T'' = T diag(beta o Gamma) in bf16
-// The kernel is bound by the latency of the fp32 solve, so it is laid out for occupancy: 55 KB of
-// shared memory (the Q tiles are recycled for the rows being solved, A^T is kept as its ten
-// non-zero 16x16 blocks and later recycled for the T'' operand) and 128 tensor-memory columns.
+// every tensor-core product M = 128 (thread r = head (r / 64) of the pair, row r % 64):
+//   MMA1   [Q ; K] K^T           (128 x 64 x 128)  rows 0-63: Q K^T, rows 64-127: K K^T
+//   solve  T = (I + A)^-1 row by row through the transposed system y (I + A) = e_i, blocked by
+//          16 columns from the right:
+//              y_blk(jb) = (e_blk(jb) - sum_{mb > jb} y_blk(mb) A[mb][jb]) (I + A[jb][jb])^-1
+//          The sum over finished blocks is a small tensor-core product (y as bf16 hi + lo A operand
+//          in tensor memory, the off-diagonal blocks of A as bf16 hi + lo B tiles, fp32 accumulate);
+//          only the 16 x 16 diagonal solve stays in fp32 registers.  Four dependent steps instead
+//          of a 64-long substitution chain, equal work for every row.
+//   MMA2   [T''_a ; T''_b] K     (128 x 128 x 64)  T'' = T diag(beta o Gamma) in bf16
+// K K^T is symmetric, so the thread that owns row j of K K^T produces COLUMN j of A, which is a
+// row of the B tile: everything is written with 16-byte shared-memory stores.
 constexpr int kIntraThreads = 128;
 constexpr uint32_t IQ_LO = 0, IK_LO = 8192, IQ_HI = 16384, IK_HI = 24576;  // TMA tiles [64][64] bf16
-constexpr uint32_t IYS2 = IQ_LO, IYS3 = IQ_HI;  // after MMA1: columns 32-47 / 48-63 of the rows being solved, fp32 [16][128]
-constexpr uint32_t IAT = 32768;                 // A^T, two heads x ten 16x16 fp32 blocks (j-block <= m-block)
-constexpr uint32_t IT2 = IAT;                   // after the solve: T'' operand (bf16) [128][64]
-constexpr uint32_t IGAM = IAT + 2 * 10 * 1024;  // gam[2][64] | bet[2][64] | Gam[2][64] | tmp[4]
+constexpr uint32_t IDG = IQ_LO;    // after MMA1: diagonal blocks of A^T, fp32 [2 heads][4][16][16]        8 KB
+constexpr uint32_t IBT2 = IQ_HI;   // after MMA1: B tiles of column block 2 (hi 4 KB | lo 4 KB)
+constexpr uint32_t IBT = 32768;    // B tiles of column blocks 0 and 1: [jb][hi|lo] x 4 KB               16 KB
+constexpr uint32_t IT2 = IBT;      // after the solve: T'' operand (bf16) [128][64]                       16 KB
+constexpr uint32_t IGAM = IBT + 16384;  // gam[2][64] | bet[2][64] | Gam[2][64] | tmp[4]
 constexpr uint32_t IBAR = IGAM + 6 * 64 * 4 + 64;
 constexpr uint32_t kIntraSmem = IBAR + 64 + 1024;
-constexpr uint32_t ITM_D1 = 0, ITM_D2 = 0, ITM_COLS = 128;  // the W accumulator reuses the columns of [QK^T ; KK^T]
+// tensor-memory columns: [QK^T ; KK^T] first, then the solve's operands, then the W accumulator
+constexpr uint32_t ITM_D1 = 0, ITM_YHI = 0, ITM_YLO = 32, ITM_ACC = 64, ITM_D2 = 0, ITM_COLS = 128;
 
-// index of the 16x16 block (j-block jb, m-block mb >= jb) of A^T
-__device__ __forceinline__ int at_blk(int jb, int mb) { return jb * 4 - (jb * (jb - 1)) / 2 + (mb - jb); }
+__device__ __forceinline__ uint32_t intra_btile(int jb, int lo) {  // byte offset of B tile (jb, hi/lo)
+    return (jb == 2 ? IBT2 : IBT + (uint32_t)jb * 8192u) + (uint32_t)lo * 4096u;
+}
 
 __global__ void __launch_bounds__(kIntraThreads, 4)
 gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -119,13 +126,15 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     uint64_t* bar_load = reinterpret_cast<uint64_t*>(smem + IBAR);
     uint64_t* bar_mma1 = bar_load + 1;
     uint64_t* bar_mma2 = bar_load + 2;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + IBAR + 32);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + IBAR + 40);
+    uint64_t* bar_step = bar_load + 3;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + IBAR + 40);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + IBAR + 48);
 
     if (tid == 0) {
         mbar_init(bar_load, 1);
         mbar_init(bar_mma1, 1);
         mbar_init(bar_mma2, 1);
+        mbar_init(bar_step, 1);
         *abort_flag = 0;
         mbar_fence_init();
     }
@@ -198,21 +207,26 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             wsS[64 + i] = __expf(gam[hh * 64 + len - 1] - gam[tid]);
             if (i == 0) wsS[128] = Gam[hh * 64 + len - 1];
         }
-        // ---- phase A: this thread's row of [Q K^T ; K K^T]: rows 0-63 -> P, rows 64-127 -> A^T,
-        //      sixteen columns at a time (rolled: long straight-line code runs at instruction-fetch speed)
+        // ---- phase A, sixteen columns at a time (rolled: long straight-line code runs at
+        //      instruction-fetch speed).  Rows 0-63 of the accumulator are Q K^T -> P; rows 64-127 are
+        //      K K^T, and row j of it (symmetric) yields column j of A:
+        //          A[m][j] = beta_m exp(gamma_m - gamma_j) (K K^T)_jm   for m > j, else 0
+        //      (the exponent is <= 0).  Column j is row (j % 16) of B tile (j / 16); its part inside
+        //      the diagonal block goes to the fp32 diagonal blocks instead.
         {
             const int row = tid & 63;
-            float* At = reinterpret_cast<float*>(smem + IAT);
+            const int jb_own = row >> 4;
 #pragma unroll 1
             for (int q4 = 0; q4 < 4; ++q4) {
                 uint32_t r[16];
                 tmem_ld16(lane_addr + ITM_D1 + q4 * 16, r);
                 tmem_ld_wait();
 #pragma unroll 1
-                for (int e = 0; e < nh; ++e) {
+                for (int e = 0; e < 2; ++e) {
                     const float* gm = gam + e * 64 + q4 * 16;
                     const float gi = gam[e * 64 + row];
                     if (tid < 64) {
+                        if (e >= nh) continue;
                         // P row: (Q K^T)_ij exp(gamma_i - gamma_j) for j <= i (difference masked before exp)
                         uint8_t* wsP = ws + L.off_P + ((size_t)c * Hv + hq * G + 2 * p + e) * kPBytes;
 #pragma unroll
@@ -227,101 +241,107 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                             }
                             *reinterpret_cast<uint4*>(wsP + swz(row, q4 * 2 + half)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         }
-                    } else if ((row >> 4) >= q4) {
-                        // A^T[j][i] = beta_i exp(gamma_i - gamma_j) (K K^T)_ij for j < i, else 0; block (q4, row/16)
-                        float* at = At + e * 10 * 256 + at_blk(q4, row >> 4) * 256 + (row & 15);
-                        const float bi = bet[e * 64 + row];
+                    } else if (q4 >= jb_own) {
+                        const float* bm = bet + e * 64 + q4 * 16;
+                        float a[16];
 #pragma unroll
-                        for (int jl = 0; jl < 16; ++jl)
-                            at[jl * 16] = (q4 * 16 + jl < row) ? bi * __expf(gi - gm[jl]) * __uint_as_float(r[jl]) : 0.f;
-                    }
-                }
-            }
-        }
-        tc_fence_before_sync();
-        __syncthreads();  // A^T complete; the Q tiles and the [QK^T ; KK^T] accumulator are dead from here on
-
-        // ---- UT transform, row i of T = (I + A)^-1 through the transposed system
-        //      y_j = delta_ij - sum_{m > j} y_m A[m][j],
-        // in 16-column blocks from the right.  Finished columns 32..63 of the row sit in this thread's
-        // private column of ys2/ys3, columns 16..31 and the block being solved in registers.  Rows of
-        // the upper half of the chunk never reach the two right-hand blocks, so their warps skip them.
-        float yl[16], yl1[16];
-        const int top = (warp & 1) ? 3 : 1;  // highest 16-block with a nonzero entry for this warp's rows
-        {
-            const float* at = reinterpret_cast<const float*>(smem + IAT) + hh * 10 * 256;
-            float* ys2 = reinterpret_cast<float*>(smem + IYS2) + tid;
-            float* ys3 = reinterpret_cast<float*>(smem + IYS3) + tid;
+                        for (int ml = 0; ml < 16; ++ml)
+                            a[ml] = (q4 * 16 + ml > row) ? bm[ml] * __expf(gm[ml] - gi) * __uint_as_float(r[ml]) : 0.f;
+                        if (q4 == jb_own) {
+                            float4* dg = reinterpret_cast<float4*>(smem + IDG) + ((e * 4 + jb_own) * 16 + (row & 15)) * 4;
 #pragma unroll
-            for (int jj = 0; jj < 16; ++jj) yl1[jj] = 0.f;
-#pragma unroll 1
-            for (int jb = top; jb >= 0; --jb) {
-                float acc[16];
+                            for (int q = 0; q < 4; ++q) dg[q] = make_float4(a[4 * q], a[4 * q + 1], a[4 * q + 2], a[4 * q + 3]);
+                        } else {
+                            const uint32_t n = (uint32_t)(e * 16 + (row & 15));
 #pragma unroll
-                for (int jj = 0; jj < 16; ++jj) acc[jj] = 0.f;
-                // contributions of the finished blocks held in shared memory (m-blocks 3 and 2)
-#pragma unroll 1
-                for (int mb = top; mb > jb && mb >= 2; --mb) {
-                    const float* blkp = at + at_blk(jb, mb) * 256;
-                    const float* yp = (mb == 3) ? ys3 : ys2;
-#pragma unroll 1
-                    for (int mg = 0; mg < 4; ++mg) {
-                        float4 a4[16];
+                            for (int half = 0; half < 2; ++half) {
+                                uint32_t hi4[4], lo4[4];
 #pragma unroll
-                        for (int jj = 0; jj < 16; ++jj) a4[jj] = *reinterpret_cast<const float4*>(blkp + jj * 16 + mg * 4);
-                        const float y0 = yp[(mg * 4 + 0) * 128], y1 = yp[(mg * 4 + 1) * 128];
-                        const float y2 = yp[(mg * 4 + 2) * 128], y3 = yp[(mg * 4 + 3) * 128];
-#pragma unroll
-                        for (int jj = 0; jj < 16; ++jj)
-                            acc[jj] = fmaf(a4[jj].x, y0, fmaf(a4[jj].y, y1, fmaf(a4[jj].z, y2, fmaf(a4[jj].w, y3, acc[jj]))));
-                    }
-                }
-                // contribution of m-block 1 (in registers) to block 0
-                if (jb == 0) {
-                    const float* blkp = at + at_blk(0, 1) * 256;
-#pragma unroll
-                    for (int mg = 0; mg < 4; ++mg) {
-#pragma unroll
-                        for (int jj = 0; jj < 16; ++jj) {
-                            const float4 a4 = *reinterpret_cast<const float4*>(blkp + jj * 16 + mg * 4);
-                            acc[jj] = fmaf(a4.x, yl1[mg * 4], fmaf(a4.y, yl1[mg * 4 + 1],
-                                      fmaf(a4.z, yl1[mg * 4 + 2], fmaf(a4.w, yl1[mg * 4 + 3], acc[jj]))));
+                                for (int q2 = 0; q2 < 4; ++q2)
+                                    split_bf16x2(a[half * 8 + q2 * 2], a[half * 8 + q2 * 2 + 1], hi4[q2], lo4[q2]);
+                                const uint32_t off = swz(n, q4 * 2 + half);
+                                *reinterpret_cast<uint4*>(smem + intra_btile(jb_own, 0) + off) = make_uint4(hi4[0], hi4[1], hi4[2], hi4[3]);
+                                *reinterpret_cast<uint4*>(smem + intra_btile(jb_own, 1) + off) = make_uint4(lo4[0], lo4[1], lo4[2], lo4[3]);
+                            }
                         }
                     }
                 }
-                // diagonal 16x16 block, column by column from the right: once y_mm is known its
-                // contribution is pushed to every column left of it (independent FMAs, no long chain)
-                const float* ablk = at + at_blk(jb, jb) * 256;
-#pragma unroll
-                for (int mm = 15; mm >= 0; --mm) {
-                    yl[mm] = ((16 * jb + mm) == i ? 1.f : 0.f) - acc[mm];
-#pragma unroll
-                    for (int jj = 0; jj < mm; ++jj) acc[jj] = fmaf(ablk[jj * 16 + mm], yl[mm], acc[jj]);
-                }
-                if (jb == 3) {
-#pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) ys3[jj * 128] = yl[jj];
-                } else if (jb == 2) {
-#pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) ys2[jj * 128] = yl[jj];
-                } else if (jb == 1) {
-#pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) yl1[jj] = yl[jj];
-                }
             }
         }
-        __syncthreads();  // every warp is done with A^T: its space becomes the T'' operand
-        // ---- T' = T diag(beta) -> workspace (bf16 hi + lo); T'' = T' diag(Gamma) -> smem A operand (bf16)
-        {
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        __syncthreads();  // B tiles and diagonal blocks complete; the accumulator of MMA1 is dead from here on
+        tc_fence_after_sync();
+
+        // ---- the blocked solve: z[jb][.] = columns 16 jb .. 16 jb + 15 of row i of T
+        float z[4][16];
+        constexpr uint32_t IDS = umma_idesc_bf16(128, 32, false, false, false);
+#pragma unroll
+        for (int jb = 3; jb >= 0; --jb) {
+            float rhs[16];
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) rhs[jj] = ((16 * jb + jj) == i) ? 1.f : 0.f;
+            if (jb < 3) {  // subtract sum_{mb > jb} y_blk(mb) A[mb][jb], accumulated by the tensor cores
+                uint32_t d[16];
+                tmem_ld16(lane_addr + ITM_ACC + hh * 16, d);
+                tmem_ld_wait();
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) rhs[jj] -= __uint_as_float(d[jj]);
+            }
+            // diagonal block, column by column from the right: once z_mm is known its contribution is
+            // pushed to every column left of it (independent FMAs, no long chain)
+            const float* dg = reinterpret_cast<const float*>(smem + IDG) + (hh * 4 + jb) * 256;
+#pragma unroll
+            for (int mm = 15; mm >= 0; --mm) {
+                z[jb][mm] = rhs[mm];
+#pragma unroll
+                for (int jj = 0; jj < mm; ++jj) rhs[jj] = fmaf(-dg[jj * 16 + mm], z[jb][mm], rhs[jj]);
+            }
+            if (jb > 0) {
+                // this block becomes a K step of the A operand (bf16 hi + lo) for the remaining steps
+                uint32_t zh[8], zl[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) split_bf16x2(z[jb][2 * q], z[jb][2 * q + 1], zh[q], zl[q]);
+                tmem_st8(lane_addr + ITM_YHI + jb * 8, zh);
+                tmem_st8(lane_addr + ITM_YLO + jb * 8, zl);
+                tmem_st_wait();
+                tc_fence_before_sync();
+                __syncthreads();
+                if (warp == 0) {
+                    tc_fence_after_sync();
+                    const int nj = jb - 1;
+                    const uint64_t dBh = umma_desc(sb + intra_btile(nj, 0), 16, 1024);
+                    const uint64_t dBl = umma_desc(sb + intra_btile(nj, 1), 16, 1024);
+                    const uint32_t tacc = tmem_base + ITM_ACC;
+#pragma unroll
+                    for (int mb = 3; mb >= jb; --mb) {
+                        const uint32_t ah = tmem_base + ITM_YHI + mb * 8, al = tmem_base + ITM_YLO + mb * 8;
+                        umma_bf16_ts_warp(tacc, ah, dBh + mb * 2, IDS, mb < 3);
+                        umma_bf16_ts_warp(tacc, ah, dBl + mb * 2, IDS, 1);
+                        umma_bf16_ts_warp(tacc, al, dBh + mb * 2, IDS, 1);
+                    }
+                    umma_commit_warp(bar_step);
+                    ok = mbar_wait_all(bar_step, (uint32_t)((3 - jb) & 1), abort_flag);
+                }
+                ok = __syncthreads_and(ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+            }
+        }
+        if (ok) {
+            // ---- T' = T diag(beta) -> workspace (bf16 hi + lo); T'' = T' diag(Gamma) -> smem A operand
+            //      (bf16), over the B tiles, which the last step's MMAs have finished reading
             uint8_t* wsA = ws + L.off_A + ((size_t)c * Hv + h) * kABytes;
             const float* bt = bet + hh * 64;
             const float* Gm = Gam + hh * 64;
-            auto emit = [&](int c16, const float (&yv)[8]) {
+#pragma unroll
+            for (int c16 = 0; c16 < 8; ++c16) {
                 uint32_t h1[4], l1[4], h2[4];
 #pragma unroll
                 for (int q2 = 0; q2 < 4; ++q2) {
                     const int j = c16 * 8 + q2 * 2;
-                    const float a0 = yv[q2 * 2] * bt[j], a1 = yv[q2 * 2 + 1] * bt[j + 1];
+                    const float a0 = z[c16 >> 1][(c16 & 1) * 8 + q2 * 2] * bt[j];
+                    const float a1 = z[c16 >> 1][(c16 & 1) * 8 + q2 * 2 + 1] * bt[j + 1];
                     split_bf16x2(a0, a1, h1[q2], l1[q2]);
                     h2[q2] = pack_bf16x2(a0 * Gm[j], a1 * Gm[j + 1]);
                 }
@@ -330,31 +350,13 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     *reinterpret_cast<uint4*>(wsA + 8192 + swz(i, c16)) = make_uint4(l1[0], l1[1], l1[2], l1[3]);
                 }
                 *reinterpret_cast<uint4*>(smem + IT2 + swz(tid, c16)) = make_uint4(h2[0], h2[1], h2[2], h2[3]);
-            };
-            {
-                const float a[8] = {yl[0], yl[1], yl[2], yl[3], yl[4], yl[5], yl[6], yl[7]};
-                const float b[8] = {yl[8], yl[9], yl[10], yl[11], yl[12], yl[13], yl[14], yl[15]};
-                const float cc[8] = {yl1[0], yl1[1], yl1[2], yl1[3], yl1[4], yl1[5], yl1[6], yl1[7]};
-                const float d[8] = {yl1[8], yl1[9], yl1[10], yl1[11], yl1[12], yl1[13], yl1[14], yl1[15]};
-                emit(0, a);
-                emit(1, b);
-                emit(2, cc);
-                emit(3, d);
             }
-#pragma unroll 1
-            for (int c16 = 4; c16 < 8; ++c16) {
-                const float* yp = reinterpret_cast<const float*>(smem + (c16 < 6 ? IYS2 : IYS3)) + tid + ((c16 & 1) * 8) * 128;
-                float yv[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) yv[e] = (top == 3) ? yp[e * 128] : 0.f;
-                emit(c16, yv);
-            }
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
         }
-        fence_proxy_async_smem();
-        tc_fence_before_sync();
         __syncthreads();
         // ---- MMA2: W (both heads) = [T''_a ; T''_b] K, K read MN-major from the TMA tiles
-        if (warp == 0) {
+        if (ok && warp == 0) {
             tc_fence_after_sync();
             constexpr uint32_t ID2 = umma_idesc_bf16(128, 128, false, true, false);
             const uint64_t dTh = umma_desc(sb + IT2, 16, 1024);
