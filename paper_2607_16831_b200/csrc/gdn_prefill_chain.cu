@@ -30,6 +30,15 @@ namespace gdn {
 using namespace sm100;
 
 constexpr int kChainThreads = 320;
+
+// One arrival per warp: 128 threads arriving on the same mbarrier are serialised by the
+// shared-memory unit (~500 clk before the waiter sees the phase complete); the lanes are ordered
+// by the warp barrier and lane 0 arrives for all of them.
+__device__ __forceinline__ void warp_arrive(uint64_t* bar) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
+
 // shared-memory map (bytes from a 1024-byte aligned base): two stages of per-chunk operands
 constexpr uint32_t ST_T = 0;          // T'hi 8K | T'lo 8K   (bulk copy, together with W)
 constexpr uint32_t ST_W = 16384;      // W: 2 tiles [64][64]
@@ -38,7 +47,8 @@ constexpr uint32_t ST_Q = 49152;      // Q tile                        (TMA)
 constexpr uint32_t ST_K = 65536;      // K tile                        (TMA)
 constexpr uint32_t ST_P = 81920;      // P [64][64]                    (bulk copy)
 constexpr uint32_t kStageBytes = 90112;
-constexpr uint32_t OFF_BAR = 2 * kStageBytes;          // mbarriers, TMEM slot, abort flag
+constexpr uint32_t OFF_OST = 2 * kStageBytes;          // output staging tile [64 tokens][128 v] bf16              16 KB
+constexpr uint32_t OFF_BAR = OFF_OST + 16384;          // mbarriers, TMEM slot, abort flag
 constexpr uint32_t kChainSmem = OFF_BAR + 256 + 1024;  // + slack for the manual 1024-byte alignment
 constexpr uint32_t kTxA = 32768 + 16384 + 16384;       // T'+W, V, Q
 constexpr uint32_t kTxB = 16384 + 8192;                // K, P
@@ -94,7 +104,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     if (tid == 0) {
         for (int i = 0; i < B_COUNT; ++i) {
             const bool many = (i == B_DW || i == B_SHI || i == B_STM || i == B_OFREE);
-            mbar_init(bars + i, many ? 128u : 1u);
+            mbar_init(bars + i, many ? 4u : 1u);  // one arrival per warp of the arriving role
         }
         *abort_flag = 0;
         mbar_fence_init();
@@ -298,8 +308,8 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
             tmem_st_wait();
             tc_fence_before_sync();
-            mbar_arrive(bars + B_SHI);
-            mbar_arrive(bars + B_STM);
+            warp_arrive(bars + B_SHI);
+            warp_arrive(bars + B_STM);
         }
         for (int ci = 0; ci < nchunks; ++ci) {
             const int c = c_begin + ci;
@@ -340,7 +350,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
             tmem_st_wait();
             tc_fence_before_sync();
-            mbar_arrive(bars + B_DW);
+            warp_arrive(bars + B_DW);
             if (tid == 0) GDN_STAMP(c, 18);
 
             if (!mbar_wait_all(bars + B_STATE, par, abort_flag)) break;
@@ -376,7 +386,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
                 tmem_st_wait();
                 tc_fence_before_sync();
-                mbar_arrive(bars + B_SHI);
+                warp_arrive(bars + B_SHI);
                 if (tid == 0) GDN_STAMP(c, 20);
                 // ... then the fp32 state decayed by the next chunk's Gamma_L, in place (gates the next G3B)
 #pragma unroll
@@ -395,7 +405,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
                 tmem_st_wait();
                 tc_fence_before_sync();
-                mbar_arrive(bars + B_STM);
+                warp_arrive(bars + B_STM);
                 if (tid == 0) GDN_STAMP(c, 21);
             }
         }
@@ -423,7 +433,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tmem_ld32(lane_addr + TM_OB + 32, b1);
             tmem_ld_wait();
             tc_fence_before_sync();
-            mbar_arrive(bars + B_OFREE);
+            warp_arrive(bars + B_OFREE);
             if (tid == 128) GDN_STAMP(c, 26);
             // o_i = Gamma_i Oa^T[v][i] + Ob^T[v][i], packed two tokens per register
             uint32_t op[32];
@@ -439,12 +449,29 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 op[16 + j4 * 2 + 1] = pack_bf16x2(fmaf(gn.z, __uint_as_float(a1[4 * j4 + 2]), __uint_as_float(b1[4 * j4 + 2])),
                                                   fmaf(gn.w, __uint_as_float(a1[4 * j4 + 3]), __uint_as_float(b1[4 * j4 + 3])));
             }
-            uint16_t* orow = out + ((size_t)t0 * Hv + h) * kD + v;
-            const size_t ostride = (size_t)Hv * kD;
+            // Through a shared-memory tile so that the global stores are 16 bytes per lane and whole
+            // 256-byte rows per half warp (64 two-byte stores per thread kept these warps busier than
+            // the chain itself).  The named barrier covers the four output warps only; every one of
+            // them reaches it in every iteration.
+            {
+                uint16_t* ost = reinterpret_cast<uint16_t*>(smem + OFF_OST);
+                asm volatile("bar.sync 1, 128;" ::: "memory");  // the previous chunk's tile has been read
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                if (2 * j < len) orow[(size_t)(2 * j) * ostride] = (uint16_t)(op[j] & 0xffffu);
-                if (2 * j + 1 < len) orow[(size_t)(2 * j + 1) * ostride] = (uint16_t)(op[j] >> 16);
+                for (int j = 0; j < 32; ++j) {
+                    ost[(2 * j) * kD + v] = (uint16_t)(op[j] & 0xffffu);
+                    ost[(2 * j + 1) * kD + v] = (uint16_t)(op[j] >> 16);
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const int c16 = v & 15, r0 = v >> 4;
+                uint16_t* obase = out + ((size_t)t0 * Hv + h) * kD + c16 * 8;
+                const size_t ostride = (size_t)Hv * kD;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const int row = r0 + 8 * k;
+                    if (row < len)
+                        *reinterpret_cast<uint4*>(obase + (size_t)row * ostride) =
+                            *reinterpret_cast<const uint4*>(ost + row * kD + c16 * 8);
+                }
             }
             if (tid == 128) GDN_STAMP(c, 27);
         }
