@@ -379,6 +379,17 @@ def run_gpu(args):
             torch.cuda.empty_cache()
         line["decode_sweep"] = {"timing": "40 back-to-back calls in one CUDA graph, cold (rotating) state buffers",
                                 "points": sweep}
+        # ---- the same decode with the gate arithmetic fused in (raw a, b, A_log, dt_bias)
+        from gdn_inputs import make_raw_gates
+
+        cfg_g, dg, sig, sog, oog, nbg = decode_buffers(64)
+        ra, rb, rA, rdt = (torch.from_numpy(x).cuda() for x in make_raw_gates(64, 32))
+        med, mn = time_graph(lambda i: gdn.gdn_decode_gated(dg["q"], dg["k"], dg["v"], ra, rb, rA, rdt, sig[i % nbg],
+                                                            sog[i % nbg], oog), iters=40)
+        line["decode_gated_b64"] = {"us_per_call": med, "state_gbs": 64 * STATE_BYTES_PER_ITEM / med / 1e3,
+                                    "note": "gdn_decode_gated: g and beta computed in the kernel from raw gate inputs"}
+        del cfg_g, dg, sig, sog, oog
+        torch.cuda.empty_cache()
         # ---- prefill workloads
         pre = []
         reps = 5 if args.quick else 15

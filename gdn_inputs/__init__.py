@@ -35,6 +35,7 @@ __all__ = [
     "make_state",
     "make_cu_seqlens",
     "make_varlen_lengths",
+    "make_raw_gates",
     "config",
     "CONFIG_NAMES",
 ]
@@ -134,6 +135,20 @@ def make_tokens(
         dv=dv,
         meta={"seed": seed, "gate_mean": gate_mean, "key_correlation": key_correlation},
     )
+
+
+def make_raw_gates(T: int, Hv: int, seed: int = 0):
+    """Raw gate inputs of the paper's gate parameterisation: a, b fp32 [T,Hv] ~ N(0,1);
+    A_log = log(U(1,16)) and dt_bias = softplus^-1(dt), dt log-uniform in [1e-3, 1e-1], fp32 [Hv]
+    (the usual initialisation of this layer), so exp(A_log) softplus(a + dt_bias) stays within a
+    few units.  Returns (a, b, A_log, dt_bias)."""
+    rng = np.random.default_rng(seed + 15485863)
+    a = rng.standard_normal((T, Hv), dtype=np.float32)
+    b = rng.standard_normal((T, Hv), dtype=np.float32)
+    A_log = np.log(rng.uniform(1.0, 16.0, size=Hv)).astype(np.float32)
+    dt = np.exp(rng.uniform(np.log(1e-3), np.log(1e-1), size=Hv))
+    dt_bias = (dt + np.log(-np.expm1(-dt))).astype(np.float32)
+    return a, b, A_log, dt_bias
 
 
 def make_state(N: int, Hv: int, dk: int = 128, dv: int = 128, seed: int = 0, sd: float = 0.02,

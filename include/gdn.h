@@ -118,6 +118,26 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
                 void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Both entry points with the gate arithmetic fused in (Section 3.2 of the paper, its first
+ * two lines): instead of the log-decay g and the write strength beta the caller passes the raw
+ * gate inputs
+ *   a, b      fp32 [B or T_tot, Hv]     per token and value head
+ *   A_log     fp32 [Hv]                 per value head
+ *   dt_bias   fp32 [Hv]                 per value head (the paper's b_dt)
+ * and the kernels evaluate, in fp32,
+ *   alpha = exp(g),  g = -exp(A_log) * softplus(a + dt_bias),   beta = sigmoid(b).
+ * All other arguments, results and error behaviour are those of gdn_decode / gdn_prefill.
+ */
+int gdn_decode_gated(const void* q, const void* k, const void* v, const float* a, const float* b,
+                     const float* A_log, const float* dt_bias, const float* state_in, float* state_out, void* out,
+                     int B, int Hqk, int Hv, int dk, int dv, void* stream);
+int gdn_prefill_gated(const void* q, const void* k, const void* v, const float* a, const float* b,
+                      const float* A_log, const float* dt_bias, const int32_t* cu_seqlens,
+                      const float* initial_state, void* out, float* final_state,
+                      int total_tokens, int num_seqs, int max_seqlen, int Hqk, int Hv, int dk, int dv,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Token-serial prefill: the same inputs and outputs as gdn_prefill (no workspace),
  * computed by the per-token recurrence of Section 3.2 with the state rows held in
  * registers and split along V across thread blocks (the paper's own prefill shape).

@@ -44,6 +44,10 @@ def _load():
         lib.gdn_oracle_prefill.restype = I
         lib.gdn_oracle_decode.argtypes = [P] * 8 + [I] * 6
         lib.gdn_oracle_decode.restype = I
+        lib.gdn_oracle_prefill_gated.argtypes = [P] * 11 + [I] * 6
+        lib.gdn_oracle_prefill_gated.restype = I
+        lib.gdn_oracle_decode_gated.argtypes = [P] * 10 + [I] * 6
+        lib.gdn_oracle_decode_gated.restype = I
         _lib = lib
     return _lib
 
@@ -105,4 +109,45 @@ def decode(q, k, v, g, beta, state_in, threads: Optional[int] = None) -> Tuple[n
                                    _ptr(so), _ptr(out), B, Hqk, Hv, dk, dv, threads or default_threads())
     if rc != 0:
         raise ValueError("gdn_oracle_decode: bad arguments")
+    return out, so
+
+
+def prefill_gated(q, k, v, a, b, A_log, dt_bias, cu_seqlens, initial_state=None, want_final=True,
+                  threads: Optional[int] = None):
+    """As `prefill`, with the raw gate inputs: a,b fp32 [T,Hv]; A_log, dt_bias fp32 [Hv];
+    alpha = exp(-exp(A_log) softplus(a + dt_bias)), beta = sigmoid(b) in fp64."""
+    q, k, v = _c(q, np.uint16), _c(k, np.uint16), _c(v, np.uint16)
+    a, b = _c(a, np.float32), _c(b, np.float32)
+    A_log, dt_bias = _c(A_log, np.float32), _c(dt_bias, np.float32)
+    cu = _c(cu_seqlens, np.int32)
+    T, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    N = cu.shape[0] - 1
+    assert a.shape == (T, Hv) and b.shape == (T, Hv) and A_log.shape == (Hv,) and dt_bias.shape == (Hv,)
+    if initial_state is not None:
+        initial_state = _c(initial_state, np.float32)
+    out = np.zeros((T, Hv, dv), dtype=np.float64)
+    fin = np.zeros((N, Hv, dv, dk), dtype=np.float64) if want_final else None
+    rc = _load().gdn_oracle_prefill_gated(_ptr(q), _ptr(k), _ptr(v), _ptr(a), _ptr(b), _ptr(A_log), _ptr(dt_bias),
+                                          _ptr(cu), _ptr(initial_state), _ptr(out), _ptr(fin), N, Hqk, Hv, dk, dv,
+                                          threads or default_threads())
+    if rc != 0:
+        raise ValueError("gdn_oracle_prefill_gated: bad arguments")
+    return out, fin
+
+
+def decode_gated(q, k, v, a, b, A_log, dt_bias, state_in, threads: Optional[int] = None):
+    q, k, v = _c(q, np.uint16), _c(k, np.uint16), _c(v, np.uint16)
+    a, b = _c(a, np.float32), _c(b, np.float32)
+    A_log, dt_bias = _c(A_log, np.float32), _c(dt_bias, np.float32)
+    state_in = _c(state_in, np.float32)
+    B, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    out = np.zeros((B, Hv, dv), dtype=np.float64)
+    so = np.zeros((B, Hv, dv, dk), dtype=np.float64)
+    rc = _load().gdn_oracle_decode_gated(_ptr(q), _ptr(k), _ptr(v), _ptr(a), _ptr(b), _ptr(A_log), _ptr(dt_bias),
+                                         _ptr(state_in), _ptr(so), _ptr(out), B, Hqk, Hv, dk, dv,
+                                         threads or default_threads())
+    if rc != 0:
+        raise ValueError("gdn_oracle_decode_gated: bad arguments")
     return out, so

@@ -21,6 +21,9 @@
  * Inputs are the bf16/fp32 arrays the GPU receives, widened exactly to fp64.
  * No blocking, fusion or reordering beyond the five lines above.
  *
+ * The *_gated entry points take the paper's raw gate inputs (Section 3.2, first two lines:
+ * g = exp(-exp(A_log) softplus(a + b_dt)), beta = sigmoid(b)) and evaluate them in fp64.
+ *
  * Pins (tests/test_oracle_pins.py): one-token closed form, beta = 0 pure decay,
  * one-hot-key associative recall, the per-step identity for S k, the
  * orthogonal-key closed form through library matmuls, split/packing invariance,
@@ -42,7 +45,8 @@ static double bf16_to_double(uint16_t b) {
 
 typedef struct {
     const uint16_t *q, *k, *v;
-    const float *g, *beta;
+    const float *g, *beta;          /* log-decay and write strength, or (gated entry points) the raw a and b */
+    const float *A_log, *dt_bias;   /* per value head; NULL unless the raw-gate form is used */
     const int32_t *cu_seqlens; /* NULL => decode: sequence n is the single token n */
     const float *initial_state;
     double *out, *final_state;
@@ -71,8 +75,17 @@ static void run_unit(const job_t *J, int n, int h, double *S, double *kk, double
             kk[c] = bf16_to_double(kt[c]);
             qq[c] = bf16_to_double(qt[c]);
         }
-        const double alpha = exp((double)J->g[(size_t)t * Hv + h]);
-        const double beta = (double)J->beta[(size_t)t * Hv + h];
+        double alpha, beta;
+        if (J->A_log) {
+            /* Section 3.2, first two lines: g = exp(-exp(A_log) softplus(a + dt_bias)), beta = sigmoid(b) */
+            const double x = (double)J->g[(size_t)t * Hv + h] + (double)J->dt_bias[h];
+            const double softplus = (x > 0.0 ? x : 0.0) + log1p(exp(-fabs(x)));
+            alpha = exp(-exp((double)J->A_log[h]) * softplus);
+            beta = 1.0 / (1.0 + exp(-(double)J->beta[(size_t)t * Hv + h]));
+        } else {
+            alpha = exp((double)J->g[(size_t)t * Hv + h]);
+            beta = (double)J->beta[(size_t)t * Hv + h];
+        }
         double *o = J->out + ((size_t)t * Hv + h) * dv;
         for (int r = 0; r < dv; ++r) {
             double *Sr = S + (size_t)r * dk;
@@ -156,5 +169,38 @@ int gdn_oracle_decode(const uint16_t *q, const uint16_t *k, const uint16_t *v, c
     J.out = out; J.final_state = state_out;
     J.num_seqs = B; J.Hqk = Hqk; J.Hv = Hv; J.dk = dk; J.dv = dv;
     if (!state_in) return 1;
+    return run_job(&J, num_threads);
+}
+
+/* Raw-gate forms (Section 3.2): a, b fp32 [T,Hv]; A_log, dt_bias fp32 [Hv];
+ * alpha = exp(-exp(A_log) softplus(a + dt_bias)), beta = sigmoid(b), evaluated in fp64. */
+int gdn_oracle_prefill_gated(const uint16_t *q, const uint16_t *k, const uint16_t *v, const float *a,
+                             const float *b, const float *A_log, const float *dt_bias,
+                             const int32_t *cu_seqlens, const float *initial_state, double *out,
+                             double *final_state, int num_seqs, int Hqk, int Hv, int dk, int dv,
+                             int num_threads) {
+    job_t J;
+    memset(&J, 0, sizeof J);
+    J.q = q; J.k = k; J.v = v; J.g = a; J.beta = b; J.A_log = A_log; J.dt_bias = dt_bias;
+    J.cu_seqlens = cu_seqlens;
+    J.initial_state = initial_state;
+    J.out = out; J.final_state = final_state;
+    J.num_seqs = num_seqs; J.Hqk = Hqk; J.Hv = Hv; J.dk = dk; J.dv = dv;
+    if (!cu_seqlens || !A_log || !dt_bias) return 1;
+    return run_job(&J, num_threads);
+}
+
+int gdn_oracle_decode_gated(const uint16_t *q, const uint16_t *k, const uint16_t *v, const float *a,
+                            const float *b, const float *A_log, const float *dt_bias,
+                            const float *state_in, double *state_out, double *out, int B, int Hqk,
+                            int Hv, int dk, int dv, int num_threads) {
+    job_t J;
+    memset(&J, 0, sizeof J);
+    J.q = q; J.k = k; J.v = v; J.g = a; J.beta = b; J.A_log = A_log; J.dt_bias = dt_bias;
+    J.cu_seqlens = NULL;
+    J.initial_state = state_in;
+    J.out = out; J.final_state = state_out;
+    J.num_seqs = B; J.Hqk = Hqk; J.Hv = Hv; J.dk = dk; J.dv = dv;
+    if (!state_in || !A_log || !dt_bias) return 1;
     return run_job(&J, num_threads);
 }

@@ -20,6 +20,7 @@ STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL", 2: "GDN_ERR_SHAPE", 3: "GDN_ERR_
 # Every symbol include/gdn.h declares.
 EXPORTS = ("gdn_status_string", "gdn_decode", "gdn_decode_variant", "gdn_decode_num_variants",
            "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_recurrent", "gdn_prefill_static",
+           "gdn_decode_gated", "gdn_prefill_gated",
            "gdn_last_device_status")
 
 
@@ -57,6 +58,10 @@ def lib() -> ctypes.CDLL:
         L.gdn_prefill_recurrent.restype = I
         L.gdn_prefill_static.argtypes = [P] * 9 + [I] * 7 + [P]
         L.gdn_prefill_static.restype = I
+        L.gdn_decode_gated.argtypes = [P] * 10 + [I] * 5 + [P]
+        L.gdn_decode_gated.restype = I
+        L.gdn_prefill_gated.argtypes = [P] * 11 + [I] * 7 + [P, Z, P]
+        L.gdn_prefill_gated.restype = I
         L.gdn_last_device_status.argtypes = [P, ctypes.POINTER(I), P]
         L.gdn_last_device_status.restype = I
         _lib = L
@@ -131,6 +136,29 @@ def gdn_prefill_recurrent(q, k, v, g, beta, cu_seqlens, initial_state, out, fina
                                      _ptr(initial_state), _ptr(out), _ptr(final_state), T, N, int(max_seqlen),
                                      Hqk, Hv, dk, dv, _stream(stream))
     _check(rc, "gdn_prefill_recurrent")
+
+
+def gdn_decode_gated(q, k, v, a, b, A_log, dt_bias, state_in, state_out, out, stream=None) -> None:
+    """gdn_decode with the gate arithmetic fused in: a,b fp32 [B,Hv] raw gate inputs, A_log and
+    dt_bias fp32 [Hv]; alpha = exp(-exp(A_log) softplus(a + dt_bias)), beta = sigmoid(b)."""
+    B, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    rc = lib().gdn_decode_gated(_ptr(q), _ptr(k), _ptr(v), _ptr(a), _ptr(b), _ptr(A_log), _ptr(dt_bias),
+                                _ptr(state_in), _ptr(state_out), _ptr(out), B, Hqk, Hv, dk, dv, _stream(stream))
+    _check(rc, "gdn_decode_gated")
+
+
+def gdn_prefill_gated(q, k, v, a, b, A_log, dt_bias, cu_seqlens, initial_state, out, final_state, max_seqlen: int,
+                      workspace, stream=None) -> None:
+    """gdn_prefill with the gate arithmetic fused in (see gdn_decode_gated)."""
+    T, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    N = cu_seqlens.shape[0] - 1
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().gdn_prefill_gated(_ptr(q), _ptr(k), _ptr(v), _ptr(a), _ptr(b), _ptr(A_log), _ptr(dt_bias),
+                                 _ptr(cu_seqlens), _ptr(initial_state), _ptr(out), _ptr(final_state), T, N,
+                                 int(max_seqlen), Hqk, Hv, dk, dv, _ptr(workspace), wbytes, _stream(stream))
+    _check(rc, "gdn_prefill_gated")
 
 
 PREFILL_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024

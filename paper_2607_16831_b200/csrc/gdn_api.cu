@@ -6,15 +6,16 @@
 
 namespace gdn {
 cudaError_t decode_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
-                            const float* s_in, float* s_out, void* out, int B, int Hqk, int Hv, int variant,
-                            cudaStream_t st);
+                            const float* A_log, const float* dt_bias, const float* s_in, float* s_out, void* out,
+                            int B, int Hqk, int Hv, int variant, cudaStream_t st);
 cudaError_t prefill_recurrent_dispatch(const void* q, const void* k, const void* v, const float* g,
                                        const float* beta, const int32_t* cu_seqlens, const float* initial_state,
                                        void* out, float* final_state, int total_tokens, int num_seqs, int Hqk,
                                        int Hv, cudaStream_t st);
 size_t prefill_chunked_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv);
 cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v, const float* g,
-                                     const float* beta, const int32_t* cu_seqlens, const float* initial_state,
+                                     const float* beta, const float* A_log, const float* dt_bias,
+                                     const int32_t* cu_seqlens, const float* initial_state,
                                      void* out, float* final_state, int total_tokens, int num_seqs,
                                      int max_seqlen, int Hqk, int Hv, void* workspace, size_t workspace_bytes,
                                      cudaStream_t st);
@@ -53,19 +54,21 @@ static int check_heads(int Hqk, int Hv, int dk, int dv) {
 }
 
 static int decode_impl(const void* q, const void* k, const void* v, const float* g, const float* beta,
-                       const float* state_in, float* state_out, void* out, int B, int Hqk, int Hv, int dk, int dv,
-                       int variant, void* stream) {
+                       const float* A_log, const float* dt_bias, bool gated, const float* state_in, float* state_out,
+                       void* out, int B, int Hqk, int Hv, int dk, int dv, int variant, void* stream) {
     if (B < 0) return GDN_ERR_SHAPE;
     if (int rc = check_heads(Hqk, Hv, dk, dv)) return rc;
     if (B == 0) return GDN_OK;
     if (!q || !k || !v || !g || !beta || !state_in || !state_out || !out) return GDN_ERR_NULL;
+    if (gated && (!A_log || !dt_bias)) return GDN_ERR_NULL;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
-        !aligned16(state_in) || !aligned16(state_out) || !aligned16(out))
+        !aligned16(state_in) || !aligned16(state_out) || !aligned16(out) ||
+        (reinterpret_cast<uintptr_t>(A_log) & 3u) || (reinterpret_cast<uintptr_t>(dt_bias) & 3u))
         return GDN_ERR_ALIGN;
     if ((long long)B * Hv * 32 > 0x7fffffffLL) return GDN_ERR_SHAPE;
     if (!device_supported()) return GDN_ERR_UNSUPPORTED;
-    return cuda_status(decode_dispatch(q, k, v, g, beta, state_in, state_out, out, B, Hqk, Hv, variant,
-                                       (cudaStream_t)stream), "gdn_decode");
+    return cuda_status(decode_dispatch(q, k, v, g, beta, gated ? A_log : nullptr, gated ? dt_bias : nullptr, state_in,
+                                       state_out, out, B, Hqk, Hv, variant, (cudaStream_t)stream), "gdn_decode");
 }
 
 static int check_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
@@ -112,14 +115,16 @@ const char* gdn_status_string(int status) {
 int gdn_decode(const void* q, const void* k, const void* v, const float* g, const float* beta,
                const float* state_in, float* state_out, void* out, int B, int Hqk, int Hv, int dk, int dv,
                void* stream) {
-    return decode_impl(q, k, v, g, beta, state_in, state_out, out, B, Hqk, Hv, dk, dv, -1, stream);
+    return decode_impl(q, k, v, g, beta, nullptr, nullptr, false, state_in, state_out, out, B, Hqk, Hv, dk, dv, -1,
+                       stream);
 }
 
 int gdn_decode_variant(const void* q, const void* k, const void* v, const float* g, const float* beta,
                        const float* state_in, float* state_out, void* out, int B, int Hqk, int Hv, int dk, int dv,
                        int variant, void* stream) {
     if (variant < 0 || variant >= gdn_decode_num_variants()) return GDN_ERR_SHAPE;
-    return decode_impl(q, k, v, g, beta, state_in, state_out, out, B, Hqk, Hv, dk, dv, variant, stream);
+    return decode_impl(q, k, v, g, beta, nullptr, nullptr, false, state_in, state_out, out, B, Hqk, Hv, dk, dv, variant,
+                       stream);
 }
 
 int gdn_decode_num_variants(void) { return 10; }
@@ -142,9 +147,35 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
     const size_t need = prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
         return GDN_ERR_WORKSPACE;
-    return cuda_status(prefill_chunked_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
-                                                total_tokens, num_seqs, max_seqlen, Hqk, Hv, workspace,
+    return cuda_status(prefill_chunked_dispatch(q, k, v, g, beta, nullptr, nullptr, cu_seqlens, initial_state, out,
+                                                final_state, total_tokens, num_seqs, max_seqlen, Hqk, Hv, workspace,
                                                 workspace_bytes, (cudaStream_t)stream), "gdn_prefill");
+}
+
+int gdn_decode_gated(const void* q, const void* k, const void* v, const float* a, const float* b, const float* A_log,
+                     const float* dt_bias, const float* state_in, float* state_out, void* out, int B, int Hqk,
+                     int Hv, int dk, int dv, void* stream) {
+    return decode_impl(q, k, v, a, b, A_log, dt_bias, true, state_in, state_out, out, B, Hqk, Hv, dk, dv, -1, stream);
+}
+
+int gdn_prefill_gated(const void* q, const void* k, const void* v, const float* a, const float* b,
+                      const float* A_log, const float* dt_bias, const int32_t* cu_seqlens,
+                      const float* initial_state, void* out, float* final_state, int total_tokens, int num_seqs,
+                      int max_seqlen, int Hqk, int Hv, int dk, int dv, void* workspace, size_t workspace_bytes,
+                      void* stream) {
+    bool nothing = false;
+    if (int rc = check_prefill(q, k, v, a, b, cu_seqlens, initial_state, out, final_state, total_tokens, num_seqs,
+                               max_seqlen, Hqk, Hv, dk, dv, &nothing))
+        return rc;
+    if (nothing) return GDN_OK;
+    if (!A_log || !dt_bias) return GDN_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(A_log) & 3u) || (reinterpret_cast<uintptr_t>(dt_bias) & 3u)) return GDN_ERR_ALIGN;
+    const size_t need = prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv);
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
+        return GDN_ERR_WORKSPACE;
+    return cuda_status(prefill_chunked_dispatch(q, k, v, a, b, A_log, dt_bias, cu_seqlens, initial_state, out,
+                                                final_state, total_tokens, num_seqs, max_seqlen, Hqk, Hv, workspace,
+                                                workspace_bytes, (cudaStream_t)stream), "gdn_prefill_gated");
 }
 
 int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const float* g, const float* beta,

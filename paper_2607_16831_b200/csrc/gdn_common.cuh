@@ -41,6 +41,15 @@ __device__ __forceinline__ void split_bf16x2(float y0, float y1, uint32_t& hi, u
     lo = pack_bf16x2(y0 - h0, y1 - h1);
 }
 
+// Raw gate parameterisation (Section 3.2 of the paper, first two lines), evaluated in fp32:
+//   log-decay g = -exp(A_log) * softplus(a + dt_bias),   beta = sigmoid(b).
+__device__ __forceinline__ void raw_gates(float a, float b, float A_log, float dt_bias, float& g, float& beta) {
+    const float x = a + dt_bias;
+    const float sp = fmaxf(x, 0.f) + log1pf(__expf(-fabsf(x)));
+    g = -__expf(A_log) * sp;
+    beta = 1.f / (1.f + __expf(-b));
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace gdn

@@ -72,7 +72,8 @@ template <int NB, int WARPS>
 __global__ void __launch_bounds__(WARPS * 32)
 gdn_decode_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
                   const uint16_t* __restrict__ v, const float* __restrict__ g,
-                  const float* __restrict__ beta, const float* s_in, float* s_out,
+                  const float* __restrict__ beta, const float* __restrict__ A_log,
+                  const float* __restrict__ dt_bias, const float* s_in, float* s_out,
                   uint16_t* __restrict__ out, int Hqk, int Hv, int split) {
     const int cta = blockIdx.x;
     const int part = cta % split;
@@ -97,8 +98,10 @@ gdn_decode_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k
         unpack_bf16x2(qw.x, qf[4 * j + 0], qf[4 * j + 1]);
         unpack_bf16x2(qw.y, qf[4 * j + 2], qf[4 * j + 3]);
     }
-    const float alpha = __expf(__ldg(g + bh));
-    const float bt = __ldg(beta + bh);
+    // g/beta hold the log-decay and write strength, or (A_log != NULL) the raw gate inputs a and b
+    float gl = __ldg(g + bh), bt = __ldg(beta + bh);
+    if (A_log) raw_gates(gl, bt, __ldg(A_log + h), __ldg(dt_bias + h), gl, bt);
+    const float alpha = __expf(gl);
     float qk = 0.f;
 #pragma unroll
     for (int j = 0; j < 16; ++j) qk = fmaf(qf[j], kf[j], qk);
@@ -112,13 +115,13 @@ gdn_decode_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k
 
 template <int NB, int WARPS>
 static cudaError_t launch(const void* q, const void* k, const void* v, const float* g, const float* beta,
-                          const float* s_in, float* s_out, void* out, int B, int Hqk, int Hv,
-                          cudaStream_t st) {
+                          const float* A_log, const float* dt_bias, const float* s_in, float* s_out, void* out,
+                          int B, int Hqk, int Hv, cudaStream_t st) {
     constexpr int split = kD / (WARPS * 4 * NB);
     static_assert(split >= 1 && split * WARPS * 4 * NB == kD, "rows must tile the head");
     const long long ctas = (long long)B * Hv * split;
     gdn_decode_kernel<NB, WARPS><<<(unsigned)ctas, WARPS * 32, 0, st>>>(
-        (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta, s_in, s_out, (uint16_t*)out,
+        (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta, A_log, dt_bias, s_in, s_out, (uint16_t*)out,
         Hqk, Hv, split);
     return cudaGetLastError();
 }
@@ -127,24 +130,24 @@ static cudaError_t launch(const void* q, const void* k, const void* v, const flo
 // kernel is latency bound and wants as many small CTAs as possible (one warp, four
 // rows: 1024 CTAs at B = 1); large batches want more bytes in flight per warp.
 cudaError_t decode_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
-                            const float* s_in, float* s_out, void* out, int B, int Hqk, int Hv,
-                            int variant, cudaStream_t st) {
+                            const float* A_log, const float* dt_bias, const float* s_in, float* s_out, void* out,
+                            int B, int Hqk, int Hv, int variant, cudaStream_t st) {
     if (variant < 0) {
         if (B <= 2) variant = 0;
         else if (B <= 16) variant = 1;
         else variant = 3;
     }
     switch (variant) {
-        case 0: return launch<1, 1>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
-        case 1: return launch<2, 1>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
-        case 2: return launch<2, 2>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
-        case 3: return launch<2, 4>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
-        case 4: return launch<4, 2>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
-        case 5: return launch<4, 4>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
-        case 6: return launch<4, 8>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
-        case 7: return launch<8, 4>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
-        case 8: return launch<1, 4>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
-        case 9: return launch<2, 8>(q, k, v, g, beta, s_in, s_out, out, B, Hqk, Hv, st);
+        case 0: return launch<1, 1>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
+        case 1: return launch<2, 1>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
+        case 2: return launch<2, 2>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
+        case 3: return launch<2, 4>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
+        case 4: return launch<4, 2>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
+        case 5: return launch<4, 4>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
+        case 6: return launch<4, 8>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
+        case 7: return launch<8, 4>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
+        case 8: return launch<1, 4>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
+        case 9: return launch<2, 8>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
         default: return cudaErrorInvalidValue;
     }
 }

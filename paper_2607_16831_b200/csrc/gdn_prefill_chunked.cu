@@ -38,7 +38,8 @@ static bool make_map(CUtensorMap* m, const void* base, int T, int H) {
 }
 
 cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v, const float* g,
-                                     const float* beta, const int32_t* cu_seqlens, const float* initial_state,
+                                     const float* beta, const float* A_log, const float* dt_bias,
+                                     const int32_t* cu_seqlens, const float* initial_state,
                                      void* out, float* final_state, int total_tokens, int num_seqs,
                                      int /*max_seqlen*/, int Hqk, int Hv, void* workspace, size_t /*workspace_bytes*/,
                                      cudaStream_t st) {
@@ -51,7 +52,7 @@ cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v
         if (!make_map(&mq, q, total_tokens, Hqk) || !make_map(&mk, k, total_tokens, Hqk) ||
             !make_map(&mv, v, total_tokens, Hv))
             return cudaErrorUnknown;
-        e = launch_prefill_intra(mq, mk, g, beta, ws, L, Hqk, Hv, st);
+        e = launch_prefill_intra(mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv, st);
         if (e != cudaSuccess) return e;
         e = launch_prefill_chain(mq, mk, mv, initial_state, out, final_state, ws, L, num_seqs, Hqk, Hv, st);
         if (e != cudaSuccess) return e;

@@ -101,8 +101,9 @@ __device__ __forceinline__ uint32_t intra_btile(int jb, int lo) {  // byte offse
 
 __global__ void __launch_bounds__(kIntraThreads, 4)
 gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                         const float* __restrict__ g, const float* __restrict__ beta, uint8_t* __restrict__ ws,
-                         WsLayout L, int Hqk, int Hv) {
+                         const float* __restrict__ g, const float* __restrict__ beta,
+                         const float* __restrict__ A_log, const float* __restrict__ dt_bias,
+                         uint8_t* __restrict__ ws, WsLayout L, int Hqk, int Hv) {
     const int c = blockIdx.x;
     const int* hdr = reinterpret_cast<const int*>(ws);
     if (c >= hdr[1]) return;
@@ -169,6 +170,8 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         if (head_ok && i < len) {
             x = __ldg(g + (size_t)(t0 + i) * Hv + h);
             b = __ldg(beta + (size_t)(t0 + i) * Hv + h);
+            // with A_log given, g/beta are the raw gate inputs a and b
+            if (A_log) raw_gates(x, b, __ldg(A_log + h), __ldg(dt_bias + h), x, b);
         }
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -410,7 +413,8 @@ cudaError_t launch_prefill_prep(const int32_t* cu_seqlens, int num_seqs, int tot
 }
 
 cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, const float* g, const float* beta,
-                                 uint8_t* ws, const WsLayout& L, int Hqk, int Hv, cudaStream_t st) {
+                                 const float* A_log, const float* dt_bias, uint8_t* ws, const WsLayout& L, int Hqk,
+                                 int Hv, cudaStream_t st) {
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(gdn_prefill_intra_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -420,7 +424,7 @@ cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, c
     }
     const int G = Hv / Hqk;
     dim3 grid(L.nc_max, Hqk * ((G + 1) / 2));
-    gdn_prefill_intra_kernel<<<grid, kIntraThreads, kIntraSmem, st>>>(mq, mk, g, beta, ws, L, Hqk, Hv);
+    gdn_prefill_intra_kernel<<<grid, kIntraThreads, kIntraSmem, st>>>(mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv);
     return cudaGetLastError();
 }
 

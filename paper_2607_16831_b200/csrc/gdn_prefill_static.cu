@@ -6,7 +6,8 @@
 namespace gdn {
 size_t prefill_chunked_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv);
 cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v, const float* g,
-                                     const float* beta, const int32_t* cu_seqlens, const float* initial_state,
+                                     const float* beta, const float* A_log, const float* dt_bias,
+                                     const int32_t* cu_seqlens, const float* initial_state,
                                      void* out, float* final_state, int total_tokens, int num_seqs,
                                      int max_seqlen, int Hqk, int Hv, void* workspace, size_t workspace_bytes,
                                      cudaStream_t st);
@@ -54,7 +55,7 @@ extern "C" int gdn_prefill_static(const void* q, const void* k, const void* v, c
         if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return GDN_ERR_CUDA;
         g_static_scratch_addr[dev] = ptr;
     }
-    cudaError_t e = prefill_chunked_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
+    cudaError_t e = prefill_chunked_dispatch(q, k, v, g, beta, nullptr, nullptr, cu_seqlens, initial_state, out, final_state,
                                              total_tokens, num_seqs, max_seqlen, Hqk, Hv, g_static_scratch_addr[dev],
                                              (size_t)GDN_PREFILL_STATIC_SCRATCH_BYTES, (cudaStream_t)stream);
     return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;

@@ -51,7 +51,8 @@ __host__ __device__ __forceinline__ uint32_t swz(uint32_t r, uint32_t c16) {
 cudaError_t launch_prefill_prep(const int32_t* cu_seqlens, int num_seqs, int total_tokens, uint8_t* ws,
                                 const WsLayout& L, cudaStream_t st);
 cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, const float* g, const float* beta,
-                                 uint8_t* ws, const WsLayout& L, int Hqk, int Hv, cudaStream_t st);
+                                 const float* A_log, const float* dt_bias, uint8_t* ws, const WsLayout& L, int Hqk,
+                                 int Hv, cudaStream_t st);
 cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                                  const float* initial_state, void* out, float* final_state, uint8_t* ws,
                                  const WsLayout& L, int num_seqs, int Hqk, int Hv, cudaStream_t st);

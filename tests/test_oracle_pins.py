@@ -290,3 +290,37 @@ def test_thread_count_does_not_change_results():
     b = oracle.prefill(tok.q, tok.k, tok.v, tok.g, tok.beta, cu, init, threads=5)
     np.testing.assert_array_equal(a[0], b[0])
     np.testing.assert_array_equal(a[1], b[1])
+
+
+# ---- raw-gate form (Section 3.2): g = exp(-exp(A_log) softplus(a + dt_bias)), beta = sigmoid(b)
+def test_gated_oracle_closed_forms_and_agreement_with_the_ungated_form():
+    from gdn_inputs import make_raw_gates
+    tok = make_tokens(12, 1, 2, dk=8, dv=4, seed=100)
+    a, b, A_log, dt_bias = make_raw_gates(12, 2, seed=100)
+    init = make_state(1, 2, 8, 4, seed=100, sd=0.3)
+    cu = make_cu_seqlens([12])
+    # closed forms: a + dt_bias = 0 -> softplus = ln 2, so alpha = exp(-A ln 2) = 2^-A; b = 0 -> beta = 1/2
+    a0 = np.zeros_like(a) - dt_bias[None, :]
+    A_two = np.log(np.array([1.0, 3.0], dtype=np.float32)).astype(np.float32)
+    o, s = oracle.prefill_gated(tok.q, tok.k, tok.v, a0, np.zeros_like(b), A_two, dt_bias, cu, init)
+    alpha = np.broadcast_to(np.array([0.5, 0.125]), (12, 2))
+    # dt_bias is fp32 and a0 = -dt_bias exactly, so a + dt_bias is exactly 0
+    o2, s2 = oracle.prefill(tok.q, tok.k, tok.v, np.log(alpha).astype(np.float32), np.full((12, 2), 0.5, np.float32), cu, init)
+    assert rel_fro(o, o2) < 1e-7 and rel_fro(s, s2) < 1e-7   # only log(0.5) rounded to fp32 differs
+    # general inputs: gates computed here in fp64 with library functions, rounded to fp32, fed to the ungated form
+    x = a.astype(np.float64) + dt_bias.astype(np.float64)[None, :]
+    g64 = -np.exp(A_log.astype(np.float64))[None, :] * np.logaddexp(0.0, x)
+    beta64 = 1.0 / (1.0 + np.exp(-b.astype(np.float64)))
+    o3, s3 = oracle.prefill_gated(tok.q, tok.k, tok.v, a, b, A_log, dt_bias, cu, init)
+    o4, s4 = oracle.prefill(tok.q, tok.k, tok.v, g64.astype(np.float32), beta64.astype(np.float32), cu, init)
+    assert rel_fro(o3, o4) < 1e-6 and rel_fro(s3, s4) < 1e-6
+    # extremes: very negative a + dt_bias -> no decay; very positive b -> beta -> 1
+    o5, s5 = oracle.prefill_gated(tok.q, tok.k, tok.v, np.full_like(a, -80.0), np.full_like(b, 80.0), A_log, dt_bias, cu, init)
+    o6, s6 = oracle.prefill(tok.q, tok.k, tok.v, np.zeros_like(a), np.ones_like(b), cu, init)
+    assert rel_fro(o5, o6) < 1e-12 and rel_fro(s5, s6) < 1e-12
+    # decode form agrees with a one-token prefill
+    st = make_state(12, 2, 8, 4, seed=101, sd=0.3)
+    od, sd = oracle.decode_gated(tok.q, tok.k, tok.v, a, b, A_log, dt_bias, st)
+    op, sp = oracle.prefill_gated(tok.q, tok.k, tok.v, a, b, A_log, dt_bias, make_cu_seqlens([1] * 12), st)
+    np.testing.assert_array_equal(od, op)
+    np.testing.assert_array_equal(sd, sp)
