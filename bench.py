@@ -390,6 +390,26 @@ def run_gpu(args):
                                     "note": "gdn_decode_gated: g and beta computed in the kernel from raw gate inputs"}
         del cfg_g, dg, sig, sog, oog
         torch.cuda.empty_cache()
+        # ---- multi-token decode: T = 4 tokens per item in one pass over the state
+        from gdn_inputs import make_state, make_tokens
+
+        Tm = 4
+        tokm = make_tokens(64 * Tm, 16, 32, seed=5)
+        dm = harness.to_device(tokm)
+        stm = torch.from_numpy(make_state(64, 32, seed=5)).cuda()
+        nbm = 3
+        sim = [stm.clone() for _ in range(nbm)]
+        som = [torch.empty_like(stm) for _ in range(nbm)]
+        om = torch.empty((64, Tm, 32, 128), dtype=torch.bfloat16, device="cuda")
+        qm, km, vm = dm["q"].view(64, Tm, 16, 128), dm["k"].view(64, Tm, 16, 128), dm["v"].view(64, Tm, 32, 128)
+        gm_, bm_ = dm["g"].view(64, Tm, 32), dm["beta"].view(64, Tm, 32)
+        med, mn = time_graph(lambda i: gdn.gdn_decode_multi(qm, km, vm, gm_, bm_, sim[i % nbm], som[i % nbm], om),
+                             iters=30)
+        line["decode_multi_b64_t4"] = {"us_per_call": med, "tokens_per_s": 64 * Tm / (med * 1e-6),
+                                       "state_gbs": 64 * STATE_BYTES_PER_ITEM / med / 1e3,
+                                       "note": "gdn_decode_multi: 4 tokens per item, state read and written once"}
+        del sim, som, stm
+        torch.cuda.empty_cache()
         # ---- prefill workloads
         pre = []
         reps = 5 if args.quick else 15

@@ -79,6 +79,22 @@ int gdn_decode_variant(const void* q, const void* k, const void* v, const float*
 int gdn_decode_num_variants(void);
 
 /*
+ * Multi-token decode (the "multi-token decode" regime of Section 5.4's dispatch discussion):
+ * T tokens per batch item, applied in order by the per-token recurrence of Section 3.2 to state
+ * rows held in registers, so the state is still read once and written once per call.
+ *
+ *   q, k      bf16 [B, T, Hqk, dk]
+ *   v, out    bf16 [B, T, Hv, dv]
+ *   g, beta   fp32 [B, T, Hv]
+ *   state_in / state_out  fp32 [B, Hv, dv, dk]   (may alias exactly)
+ *
+ * T = 0 copies state_in to state_out; T = 1 is gdn_decode.
+ */
+int gdn_decode_multi(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                     const float* state_in, float* state_out, void* out,
+                     int B, int T, int Hqk, int Hv, int dk, int dv, void* stream);
+
+/*
  * Bytes of device scratch that gdn_prefill needs for the given sizes (host-side
  * arithmetic only; returns 0 for unsupported shapes).  The workspace holds the
  * per-chunk summaries (the chunk table, the cumulative gates, the UT-transformed

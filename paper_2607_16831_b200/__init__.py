@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL", 2: "GDN_ERR_SHAPE", 3: "GDN_ERR_
 # Every symbol include/gdn.h declares.
 EXPORTS = ("gdn_status_string", "gdn_decode", "gdn_decode_variant", "gdn_decode_num_variants",
            "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_recurrent", "gdn_prefill_static",
-           "gdn_decode_gated", "gdn_prefill_gated",
+           "gdn_decode_gated", "gdn_prefill_gated", "gdn_decode_multi",
            "gdn_last_device_status")
 
 
@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.gdn_prefill_recurrent.restype = I
         L.gdn_prefill_static.argtypes = [P] * 9 + [I] * 7 + [P]
         L.gdn_prefill_static.restype = I
+        L.gdn_decode_multi.argtypes = [P] * 8 + [I] * 6 + [P]
+        L.gdn_decode_multi.restype = I
         L.gdn_decode_gated.argtypes = [P] * 10 + [I] * 5 + [P]
         L.gdn_decode_gated.restype = I
         L.gdn_prefill_gated.argtypes = [P] * 11 + [I] * 7 + [P, Z, P]
@@ -136,6 +138,16 @@ def gdn_prefill_recurrent(q, k, v, g, beta, cu_seqlens, initial_state, out, fina
                                      _ptr(initial_state), _ptr(out), _ptr(final_state), T, N, int(max_seqlen),
                                      Hqk, Hv, dk, dv, _stream(stream))
     _check(rc, "gdn_prefill_recurrent")
+
+
+def gdn_decode_multi(q, k, v, g, beta, state_in, state_out, out, stream=None) -> None:
+    """T tokens per batch item in one pass over the state: q,k bf16 [B,T,Hqk,128]; v,out bf16
+    [B,T,Hv,128]; g,beta fp32 [B,T,Hv]; states fp32 [B,Hv,128,128]."""
+    B, T, Hqk, dk = q.shape
+    _, _, Hv, dv = v.shape
+    rc = lib().gdn_decode_multi(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(state_in), _ptr(state_out),
+                                _ptr(out), B, T, Hqk, Hv, dk, dv, _stream(stream))
+    _check(rc, "gdn_decode_multi")
 
 
 def gdn_decode_gated(q, k, v, a, b, A_log, dt_bias, state_in, state_out, out, stream=None) -> None:

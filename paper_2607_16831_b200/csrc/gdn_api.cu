@@ -8,6 +8,9 @@ namespace gdn {
 cudaError_t decode_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
                             const float* A_log, const float* dt_bias, const float* s_in, float* s_out, void* out,
                             int B, int Hqk, int Hv, int variant, cudaStream_t st);
+cudaError_t decode_multi_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                                  const float* s_in, float* s_out, void* out, int B, int T, int Hqk, int Hv,
+                                  cudaStream_t st);
 cudaError_t prefill_recurrent_dispatch(const void* q, const void* k, const void* v, const float* g,
                                        const float* beta, const int32_t* cu_seqlens, const float* initial_state,
                                        void* out, float* final_state, int total_tokens, int num_seqs, int Hqk,
@@ -128,6 +131,23 @@ int gdn_decode_variant(const void* q, const void* k, const void* v, const float*
 }
 
 int gdn_decode_num_variants(void) { return 10; }
+
+int gdn_decode_multi(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                     const float* state_in, float* state_out, void* out, int B, int T, int Hqk, int Hv, int dk,
+                     int dv, void* stream) {
+    if (B < 0 || T < 0) return GDN_ERR_SHAPE;
+    if (int rc = check_heads(Hqk, Hv, dk, dv)) return rc;
+    if (B == 0) return GDN_OK;
+    if (!state_in || !state_out) return GDN_ERR_NULL;
+    if (T > 0 && (!q || !k || !v || !g || !beta || !out)) return GDN_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
+        !aligned16(state_in) || !aligned16(state_out) || !aligned16(out))
+        return GDN_ERR_ALIGN;
+    if ((long long)B * Hv * 32 > 0x7fffffffLL || (long long)B * T > 0x7fffffffLL) return GDN_ERR_SHAPE;
+    if (!device_supported()) return GDN_ERR_UNSUPPORTED;
+    return cuda_status(decode_multi_dispatch(q, k, v, g, beta, state_in, state_out, out, B, T, Hqk, Hv,
+                                             (cudaStream_t)stream), "gdn_decode_multi");
+}
 
 size_t gdn_prefill_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv, int dk, int dv) {
     if (total_tokens < 0 || num_seqs < 0) return 0;

@@ -152,4 +152,110 @@ cudaError_t decode_dispatch(const void* q, const void* k, const void* v, const f
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Multi-token decode: T tokens per batch item (speculative / chunked decode), applied in order to
+// state rows that stay in registers, so the state is still read once and written once.
+// Layouts: q,k [B,T,Hqk,128], v,out [B,T,Hv,128], g,beta [B,T,Hv].
+template <int NB, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32)
+gdn_decode_multi_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
+                        const uint16_t* __restrict__ v, const float* __restrict__ g,
+                        const float* __restrict__ beta, const float* s_in, float* s_out,
+                        uint16_t* __restrict__ out, int T, int Hqk, int Hv, int split) {
+    const int cta = blockIdx.x;
+    const int part = cta % split;
+    const int bh = cta / split;
+    const int h = bh % Hv, b = bh / Hv;
+    const int hq = h / (Hv / Hqk);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane >> 3, c = lane & 7;
+    const int row0 = (part * WARPS + warp) * (4 * NB);
+    const size_t sbase = (size_t)bh * kD * kD;
+
+    float4 s[NB][4];
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
+        const float4* src = reinterpret_cast<const float4*>(s_in + sbase + (size_t)(row0 + i * 4 + sub) * kD);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) s[i][j] = __ldcs(src + c + 8 * j);
+    }
+    for (int t = 0; t < T; ++t) {
+        const size_t tok = (size_t)b * T + t;
+        const uint2* k4 = reinterpret_cast<const uint2*>(k + (tok * Hqk + hq) * kD);
+        const uint2* q4 = reinterpret_cast<const uint2*>(q + (tok * Hqk + hq) * kD);
+        float kf[16], qf[16];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint2 kw = __ldg(k4 + c + 8 * j);
+            const uint2 qw = __ldg(q4 + c + 8 * j);
+            unpack_bf16x2(kw.x, kf[4 * j + 0], kf[4 * j + 1]);
+            unpack_bf16x2(kw.y, kf[4 * j + 2], kf[4 * j + 3]);
+            unpack_bf16x2(qw.x, qf[4 * j + 0], qf[4 * j + 1]);
+            unpack_bf16x2(qw.y, qf[4 * j + 2], qf[4 * j + 3]);
+        }
+        const float alpha = __expf(__ldg(g + tok * Hv + h));
+        const float bt = __ldg(beta + tok * Hv + h);
+        float qk = 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) qk = fmaf(qf[j], kf[j], qk);
+#pragma unroll
+        for (int m = 1; m < 8; m <<= 1) qk += __shfl_xor_sync(0xffffffffu, qk, m);
+        const uint16_t* v_h = v + (tok * Hv + h) * kD;
+        uint16_t* o_h = out + (tok * Hv + h) * kD;
+#pragma unroll
+        for (int i = 0; i < NB; ++i) {
+            float a = 0.f, p = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                a = fmaf(s[i][j].x, kf[4 * j + 0], a);
+                a = fmaf(s[i][j].y, kf[4 * j + 1], a);
+                a = fmaf(s[i][j].z, kf[4 * j + 2], a);
+                a = fmaf(s[i][j].w, kf[4 * j + 3], a);
+                p = fmaf(s[i][j].x, qf[4 * j + 0], p);
+                p = fmaf(s[i][j].y, qf[4 * j + 1], p);
+                p = fmaf(s[i][j].z, qf[4 * j + 2], p);
+                p = fmaf(s[i][j].w, qf[4 * j + 3], p);
+            }
+#pragma unroll
+            for (int m = 1; m < 8; m <<= 1) {
+                a += __shfl_xor_sync(0xffffffffu, a, m);
+                p += __shfl_xor_sync(0xffffffffu, p, m);
+            }
+            const float delta = bt * (bf16_bits_to_float(__ldg(v_h + row0 + i * 4 + sub)) - alpha * a);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                s[i][j].x = fmaf(alpha, s[i][j].x, delta * kf[4 * j + 0]);
+                s[i][j].y = fmaf(alpha, s[i][j].y, delta * kf[4 * j + 1]);
+                s[i][j].z = fmaf(alpha, s[i][j].z, delta * kf[4 * j + 2]);
+                s[i][j].w = fmaf(alpha, s[i][j].w, delta * kf[4 * j + 3]);
+            }
+            if (c == 0) o_h[row0 + i * 4 + sub] = float_to_bf16_bits(fmaf(delta, qk, alpha * p));
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
+        float4* dst = reinterpret_cast<float4*>(s_out + sbase + (size_t)(row0 + i * 4 + sub) * kD);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) __stcs(dst + c + 8 * j, s[i][j]);
+    }
+}
+
+cudaError_t decode_multi_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                                  const float* s_in, float* s_out, void* out, int B, int T, int Hqk, int Hv,
+                                  cudaStream_t st) {
+    if (B <= 2) {
+        constexpr int NB = 1, WARPS = 1, split = kD / (WARPS * 4 * NB);
+        gdn_decode_multi_kernel<NB, WARPS><<<(unsigned)((long long)B * Hv * split), WARPS * 32, 0, st>>>(
+            (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta, s_in, s_out, (uint16_t*)out, T, Hqk,
+            Hv, split);
+    } else {
+        constexpr int NB = 2, WARPS = 4, split = kD / (WARPS * 4 * NB);
+        gdn_decode_multi_kernel<NB, WARPS><<<(unsigned)((long long)B * Hv * split), WARPS * 32, 0, st>>>(
+            (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta, s_in, s_out, (uint16_t*)out, T, Hqk,
+            Hv, split);
+    }
+    return cudaGetLastError();
+}
+
 }  // namespace gdn

@@ -112,3 +112,26 @@ def test_decode_then_prefill_state_handoff():
     dec_out = np.concatenate(outs, axis=0)
     assert harness.rel_fro(dec_out, pre["out"]) < 8e-3
     assert harness.rel_fro(s.cpu().numpy().astype(np.float64), pre["final_state"]) < 5e-3
+
+
+@pytest.mark.parametrize("B,T", [(1, 2), (3, 4), (64, 3), (2, 0)])
+def test_decode_multi_token(B, T):
+    """T tokens per item in one state pass == the oracle run over B sequences of length T."""
+    import torch
+    import paper_2607_16831_b200 as gdn
+    from gdn_inputs import make_cu_seqlens, make_state, make_tokens
+    Hqk, Hv = 16, 32
+    tok = make_tokens(B * T, Hqk, Hv, seed=100 + B + T, gate_mean=3.0)
+    st = make_state(B, Hv, seed=100 + B)
+    d = harness.to_device(tok)
+    shp = lambda x, H: x.view(B, T, H, 128)
+    s_in = torch.from_numpy(st).cuda()
+    s_out = torch.full_like(s_in, float("nan"))
+    out = torch.full((B, T, Hv, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    gdn.gdn_decode_multi(shp(d["q"], Hqk), shp(d["k"], Hqk), shp(d["v"], Hv), d["g"].view(B, T, Hv),
+                         d["beta"].view(B, T, Hv), s_in, s_out, out)
+    torch.cuda.synchronize()
+    ref_o, ref_s = oracle.prefill(tok.q, tok.k, tok.v, tok.g, tok.beta, make_cu_seqlens([T] * B), st)
+    got_o = harness.bf16_to_numpy(out).reshape(B * T, Hv, 128)
+    e = harness.assert_close(got_o, ref_o, s_out.cpu().numpy().astype(np.float64), ref_s, "decode multi B=%d T=%d" % (B, T))
+    assert e["state_rel_fro"] < 2e-6
