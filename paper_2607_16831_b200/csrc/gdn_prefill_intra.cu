@@ -89,8 +89,8 @@ constexpr uint32_t IDG = IQ_LO;    // after MMA1: diagonal blocks of A^T, fp32 [
 constexpr uint32_t IBT2 = IQ_HI;   // after MMA1: B tiles of column block 2 (hi 4 KB | lo 4 KB)
 constexpr uint32_t IBT = 32768;    // B tiles of column blocks 0 and 1: [jb][hi|lo] x 4 KB               16 KB
 constexpr uint32_t IT2 = IBT;      // after the solve: T'' operand (bf16) [128][64]                       16 KB
-constexpr uint32_t IGAM = IBT + 16384;  // gam[2][64] | bet[2][64] | Gam[2][64] | tmp[4]
-constexpr uint32_t IBAR = IGAM + 6 * 64 * 4 + 64;
+constexpr uint32_t IGAM = IBT + 16384;  // gam[2][64] | bet[2][64] | Gam[2][64] | cfP[2][64] | cfA[2][64] | tmp[4]
+constexpr uint32_t IBAR = IGAM + 10 * 64 * 4 + 64;
 constexpr uint32_t kIntraSmem = IBAR + 64 + 1024;
 // tensor-memory columns: [QK^T ; KK^T] first, then the solve's operands, then the W accumulator
 constexpr uint32_t ITM_D1 = 0, ITM_YHI = 0, ITM_YLO = 32, ITM_ACC = 64, ITM_D2 = 0, ITM_COLS = 128;
@@ -123,7 +123,9 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     float* gam = reinterpret_cast<float*>(smem + IGAM);
     float* bet = gam + 128;
     float* Gam = gam + 256;
-    float* tmp = gam + 384;
+    float* cfP = gam + 384;  // exp(gamma_{last column of j's 16-block} - gamma_j)
+    float* cfA = gam + 512;  // beta_m exp(gamma_m - gamma_{first row of m's 16-block})
+    float* tmp = gam + 640;
     uint64_t* bar_load = reinterpret_cast<uint64_t*>(smem + IBAR);
     uint64_t* bar_mma1 = bar_load + 1;
     uint64_t* bar_mma2 = bar_load + 2;
@@ -184,6 +186,12 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         gam[tid] = x;
         bet[tid] = b;
         Gam[tid] = __expf(x);
+        __syncthreads();
+        // The decay exp(gamma_i - gamma_j) between a row and a column of DIFFERENT 16-blocks factors
+        // through the block boundary with both exponents <= 0, so phase A needs one exp per
+        // (row, block) instead of one per element.
+        cfP[tid] = __expf(gam[(tid & ~15) | 15] - x);
+        cfA[tid] = b * __expf(x - gam[tid & ~15]);
     }
     if (warp == 0) {
         ok = mbar_wait_all(bar_load, 0, abort_flag);
@@ -232,24 +240,40 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         if (e >= nh) continue;
                         // P row: (Q K^T)_ij exp(gamma_i - gamma_j) for j <= i (difference masked before exp)
                         uint8_t* wsP = ws + L.off_P + ((size_t)c * Hv + hq * G + 2 * p + e) * kPBytes;
+                        float pv[16];
+                        if (q4 < jb_own && row < len) {        // whole block left of the diagonal block
+                            const float rf = __expf(gi - gam[e * 64 + q4 * 16 + 15]);
+                            const float* cf = cfP + e * 64 + q4 * 16;
+#pragma unroll
+                            for (int jl = 0; jl < 16; ++jl) pv[jl] = __uint_as_float(r[jl]) * (rf * cf[jl]);
+                        } else if (q4 == jb_own && row < len) {  // the diagonal block
+#pragma unroll
+                            for (int jl = 0; jl < 16; ++jl)
+                                pv[jl] = (q4 * 16 + jl <= row) ? __uint_as_float(r[jl]) * __expf(gi - gm[jl]) : 0.f;
+                        } else {
+#pragma unroll
+                            for (int jl = 0; jl < 16; ++jl) pv[jl] = 0.f;
+                        }
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {
                             uint32_t pk[4];
 #pragma unroll
-                            for (int q2 = 0; q2 < 4; ++q2) {
-                                const int jl = half * 8 + q2 * 2, j = q4 * 16 + jl;
-                                const float p0 = (j <= row && row < len) ? __uint_as_float(r[jl]) * __expf(gi - gm[jl]) : 0.f;
-                                const float p1 = (j + 1 <= row && row < len) ? __uint_as_float(r[jl + 1]) * __expf(gi - gm[jl + 1]) : 0.f;
-                                pk[q2] = pack_bf16x2(p0, p1);
-                            }
+                            for (int q2 = 0; q2 < 4; ++q2) pk[q2] = pack_bf16x2(pv[half * 8 + q2 * 2], pv[half * 8 + q2 * 2 + 1]);
                             *reinterpret_cast<uint4*>(wsP + swz(row, q4 * 2 + half)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         }
                     } else if (q4 >= jb_own) {
-                        const float* bm = bet + e * 64 + q4 * 16;
                         float a[16];
+                        if (q4 == jb_own) {
+                            const float* bm = bet + e * 64 + q4 * 16;
 #pragma unroll
-                        for (int ml = 0; ml < 16; ++ml)
-                            a[ml] = (q4 * 16 + ml > row) ? bm[ml] * __expf(gm[ml] - gi) * __uint_as_float(r[ml]) : 0.f;
+                            for (int ml = 0; ml < 16; ++ml)
+                                a[ml] = (q4 * 16 + ml > row) ? bm[ml] * __expf(gm[ml] - gi) * __uint_as_float(r[ml]) : 0.f;
+                        } else {
+                            const float rf = __expf(gam[e * 64 + q4 * 16] - gi);
+                            const float* cf = cfA + e * 64 + q4 * 16;
+#pragma unroll
+                            for (int ml = 0; ml < 16; ++ml) a[ml] = (rf * cf[ml]) * __uint_as_float(r[ml]);
+                        }
                         if (q4 == jb_own) {
                             float4* dg = reinterpret_cast<float4*>(smem + IDG) + ((e * 4 + jb_own) * 16 + (row & 15)) * 4;
 #pragma unroll
