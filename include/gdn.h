@@ -126,6 +126,17 @@ size_t gdn_prefill_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int 
  * A malformed cu_seqlens can give wrong results but never an out-of-range access:
  * every token index is clamped to [0, total_tokens).  total_tokens = 0 or
  * num_seqs = 0 returns GDN_OK without launching.
+ *
+ * Few long sequences (num_seqs * Hv chains that would leave most of the GPU idle) are
+ * additionally cut into up to 8 runs of chunks that advance at the same time.  The
+ * recurrence is affine in the state, S_end = S_in P + H over a run, so each run is
+ * walked from the zero state and from the identity, the runs' (P, H) pairs are joined by
+ * an associative scan, and the outputs of a run are corrected by S_in (M_t q_t).  This is
+ * the same step one level up as the chunked form that Section 5.5 describes (a summary per
+ * block of tokens, joined by dense products); the result is the same recurrence, rounded
+ * differently.
+ * The number of runs follows from num_seqs, Hv and max_seqlen; the environment variable
+ * GDN_PREFILL_MAX_SEGMENTS (1..8) lowers it, 1 switches the split off.
  */
 int gdn_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
                 const int32_t* cu_seqlens, const float* initial_state, void* out, float* final_state,

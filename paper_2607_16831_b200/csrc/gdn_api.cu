@@ -15,13 +15,13 @@ cudaError_t prefill_recurrent_dispatch(const void* q, const void* k, const void*
                                        const float* beta, const int32_t* cu_seqlens, const float* initial_state,
                                        void* out, float* final_state, int total_tokens, int num_seqs, int Hqk,
                                        int Hv, cudaStream_t st);
-size_t prefill_chunked_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv);
+size_t prefill_chunked_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv, bool allow_split);
 cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v, const float* g,
                                      const float* beta, const float* A_log, const float* dt_bias,
                                      const int32_t* cu_seqlens, const float* initial_state,
                                      void* out, float* final_state, int total_tokens, int num_seqs,
                                      int max_seqlen, int Hqk, int Hv, void* workspace, size_t workspace_bytes,
-                                     cudaStream_t st);
+                                     bool allow_split, cudaStream_t st);
 
 // 1 = sm_100 family, 0 = other, -1 = unknown yet.  Indexed by device ordinal.
 static int g_device_ok[64] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1,
@@ -152,7 +152,7 @@ int gdn_decode_multi(const void* q, const void* k, const void* v, const float* g
 size_t gdn_prefill_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv, int dk, int dv) {
     if (total_tokens < 0 || num_seqs < 0) return 0;
     if (check_heads(Hqk, Hv, dk, dv) != GDN_OK) return 0;
-    return prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv);
+    return prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv, true);
 }
 
 int gdn_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
@@ -164,12 +164,12 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
                                num_seqs, max_seqlen, Hqk, Hv, dk, dv, &nothing))
         return rc;
     if (nothing) return GDN_OK;
-    const size_t need = prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv);
+    const size_t need = prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv, true);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
         return GDN_ERR_WORKSPACE;
     return cuda_status(prefill_chunked_dispatch(q, k, v, g, beta, nullptr, nullptr, cu_seqlens, initial_state, out,
                                                 final_state, total_tokens, num_seqs, max_seqlen, Hqk, Hv, workspace,
-                                                workspace_bytes, (cudaStream_t)stream), "gdn_prefill");
+                                                workspace_bytes, true, (cudaStream_t)stream), "gdn_prefill");
 }
 
 int gdn_decode_gated(const void* q, const void* k, const void* v, const float* a, const float* b, const float* A_log,
@@ -190,12 +190,12 @@ int gdn_prefill_gated(const void* q, const void* k, const void* v, const float* 
     if (nothing) return GDN_OK;
     if (!A_log || !dt_bias) return GDN_ERR_NULL;
     if ((reinterpret_cast<uintptr_t>(A_log) & 3u) || (reinterpret_cast<uintptr_t>(dt_bias) & 3u)) return GDN_ERR_ALIGN;
-    const size_t need = prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv);
+    const size_t need = prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv, true);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
         return GDN_ERR_WORKSPACE;
     return cuda_status(prefill_chunked_dispatch(q, k, v, a, b, A_log, dt_bias, cu_seqlens, initial_state, out,
                                                 final_state, total_tokens, num_seqs, max_seqlen, Hqk, Hv, workspace,
-                                                workspace_bytes, (cudaStream_t)stream), "gdn_prefill_gated");
+                                                workspace_bytes, true, (cudaStream_t)stream), "gdn_prefill_gated");
 }
 
 int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const float* g, const float* beta,

@@ -23,6 +23,13 @@
 //   warp  8    issues every MMA (one elected lane)
 //   warp  9    issues every TMA / bulk copy, one chunk ahead of the MMAs
 // Hand-offs are mbarriers; every wait is bounded and failure unwinds through an abort flag.
+//
+// With `segs` > 1 a sequence is cut into that many runs of chunks and the runs advance at the same
+// time (the scan in gdn_prefill_scan.cu joins them).  Run 0 is the recurrence itself.  Every later
+// run has two CTAs per head: one starts from the zero state (its outputs and final state are the
+// parts that do not depend on the state entering the run), one starts from the identity with
+// v = 0 (its "outputs" are the queries carried back to the start of the run, M_t q_t, and its
+// final state is the run's transition matrix).
 #include "gdn_prefill_ws.cuh"
 #include "gdn_sm100.cuh"
 
@@ -69,9 +76,13 @@ __global__ void __launch_bounds__(kChainThreads, 1)
 gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const __grid_constant__ CUtensorMap map_v, const float* initial_state,
                          uint16_t* __restrict__ out, float* final_state, uint8_t* __restrict__ ws, WsLayout L,
-                         int Hqk, int Hv) {
-    // CTAs are handed out longest sequence first
-    const int h = blockIdx.x % Hv, n = reinterpret_cast<const int*>(ws + L.off_seq_order)[blockIdx.x / Hv];
+                         int Hqk, int Hv, int segs) {
+    // CTAs are handed out longest sequence first; within a sequence: run 0, then (zero, identity) per run
+    const int per_seq = 2 * segs - 1;
+    const int h = blockIdx.x % Hv, unit = blockIdx.x / Hv;
+    const int n = reinterpret_cast<const int*>(ws + L.off_seq_order)[unit / per_seq];
+    const int seg = (unit % per_seq + 1) >> 1;
+    const bool ident = seg > 0 && ((unit % per_seq) & 1) == 0;  // identity start, v = 0
     const int hq = h / (Hv / Hqk);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -83,11 +94,12 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
     const int* chunk_off = reinterpret_cast<const int*>(ws + L.off_chunk_off);
     const int4* chunk_info = reinterpret_cast<const int4*>(ws + L.off_chunk_info);
-    const int c_begin = chunk_off[n], c_end = chunk_off[n + 1];
-    const int nchunks = c_end - c_begin;
+    int seg_first, nchunks;
+    segment_range(chunk_off[n + 1] - chunk_off[n], segs, seg, seg_first, nchunks);
+    const int c_begin = chunk_off[n] + seg_first, c_end = c_begin + nchunks;
 
-    if (nchunks <= 0) {  // empty sequence: the state passes through
-        if (final_state && tid < kD) {
+    if (nchunks <= 0) {  // empty sequence: the state passes through; empty run: nothing to do
+        if (seg == 0 && final_state && tid < kD) {
             const size_t sb0 = ((size_t)n * Hv + h) * kD * kD + (size_t)tid * kD;
             for (int j = 0; j < kD; j += 4) {
                 float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -100,6 +112,14 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     // chunks of one sequence are consecutive: chunk ci starts at t0_first + 64 ci
     const int t0_first = chunk_info[c_begin].y;
     const int t_end = chunk_info[c_end - 1].y + chunk_info[c_end - 1].z;
+    // where this CTA's state comes from and where its results go
+    const size_t state_off = ((size_t)n * Hv + h) * kD * kD;
+    const float* init_ptr = (seg == 0 && initial_state) ? initial_state + state_off : nullptr;
+    float* fin_ptr = final_state ? final_state + state_off : nullptr;
+    if (segs > 1)
+        fin_ptr = reinterpret_cast<float*>(
+            ws + seg_block_offset(L, n, seg == 0 ? 1 : seg, h, Hv, seg == 0 ? kSegSin : (ident ? kSegP : kSegH)));
+    uint16_t* out_ptr = ident ? reinterpret_cast<uint16_t*>(ws + L.off_qt) : out;
 
     if (tid == 0) {
         for (int i = 0; i < B_COUNT; ++i) {
@@ -137,6 +157,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             const uint32_t sb = __shfl_sync(0xffffffffu, smem_u32(smem), 0);
             const uint32_t tmem_base_u = __shfl_sync(0xffffffffu, tmem_base, 0);
             const int nchunks_u = __shfl_sync(0xffffffffu, nchunks, 0);
+            const bool ident_u = __shfl_sync(0xffffffffu, (int)ident, 0) != 0;  // v = 0: no V^T T'^T term
             constexpr uint32_t ID_G1 = umma_idesc_bf16(128, 64, true, false, false);    // V^T (MN-major A) x T'^T
             constexpr uint32_t ID_G2A = umma_idesc_bf16(128, 64, false, false, true);   // -(S) x W^T
             constexpr uint32_t ID_N64 = umma_idesc_bf16(128, 64, false, false, false);  // S x Q^T ; Delta^T x P^T
@@ -174,7 +195,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 if (!g1_issued) {
                     GDN_WAIT(B_FULL_A0 + st, ph2);
                     tc_fence_after_sync();
-                    issue_G1(st);
+                    if (!ident_u) issue_G1(st);
                 }
                 g1_issued = false;
                 // ---- on the chain: Delta^T -= S W^T   (A = bf16 S in tensor memory)
@@ -185,7 +206,8 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     const uint64_t w0 = dW0 + so, w1 = dW1 + so;
                     const uint32_t td = tmem_base_u + TM_DELTA, ta = tmem_base_u + TM_SHI;
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) umma_bf16_ts_warp(td, ta + ks * 8, w0 + ks * 2, ID_G2A, 1);
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_bf16_ts_warp(td, ta + ks * 8, w0 + ks * 2, ID_G2A, (ks > 0 || !ident_u) ? 1u : 0u);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) umma_bf16_ts_warp(td, ta + 32 + ks * 8, w1 + ks * 2, ID_G2A, 1);
                 }
@@ -226,7 +248,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 if (!last) {
                     GDN_WAIT(B_FULL_A0 + (st ^ 1), ((ci + 1) >> 1) & 1);  // requested a whole chunk ago
                     tc_fence_after_sync();
-                    issue_G1(st ^ 1);
+                    if (!ident_u) issue_G1(st ^ 1);
                     g1_issued = true;
                 }
                 umma_commit_warp(bars + B_O);
@@ -273,7 +295,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         // =========================================================== chain warps
         const int v = tid;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
-        const size_t sbase = ((size_t)n * Hv + h) * kD * kD + (size_t)v * kD;
+        const size_t sbase = (size_t)v * kD;
         // initial state: bf16 operand copy and Gamma_L(first chunk) * S, both into tensor memory
         {
             const float gl0 = __ldg(scal_ptr(c_begin) + 128);
@@ -283,9 +305,13 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
                 for (int j = 0; j < 32; j += 4) {
                     float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
-                    if (initial_state) {
-                        x = *reinterpret_cast<const float4*>(initial_state + sbase + b * 64 + j);
-                        y = *reinterpret_cast<const float4*>(initial_state + sbase + b * 64 + 32 + j);
+                    if (init_ptr) {
+                        x = *reinterpret_cast<const float4*>(init_ptr + sbase + b * 64 + j);
+                        y = *reinterpret_cast<const float4*>(init_ptr + sbase + b * 64 + 32 + j);
+                    } else if (ident) {
+                        const int d0 = v - (b * 64 + j), d1 = d0 - 32;  // the one of row v sits in column v
+                        x = make_float4(d0 == 0 ? 1.f : 0.f, d0 == 1 ? 1.f : 0.f, d0 == 2 ? 1.f : 0.f, d0 == 3 ? 1.f : 0.f);
+                        y = make_float4(d1 == 0 ? 1.f : 0.f, d1 == 1 ? 1.f : 0.f, d1 == 2 ? 1.f : 0.f, d1 == 3 ? 1.f : 0.f);
                     }
                     r0[j + 0] = __float_as_uint(x.x); r0[j + 1] = __float_as_uint(x.y);
                     r0[j + 2] = __float_as_uint(x.z); r0[j + 3] = __float_as_uint(x.w);
@@ -357,7 +383,10 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tc_fence_after_sync();
             if (tid == 0) GDN_STAMP(c, 19);
             if (last) {
-                if (final_state) {
+                if (fin_ptr) {
+                    // run 0 of a split sequence also leaves its final state as the bf16 operand tiles
+                    // the fix-up of run 1 multiplies with
+                    uint8_t* img = (segs > 1 && seg == 0) ? ws + seg_block_offset(L, n, 1, h, Hv, kSegSinImg) : nullptr;
 #pragma unroll 1
                     for (int b = 0; b < 4; ++b) {
                         uint32_t r[32];
@@ -365,8 +394,17 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         tmem_ld_wait();
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<float4*>(final_state + sbase + b * 32 + j) = make_float4(
+                            *reinterpret_cast<float4*>(fin_ptr + sbase + b * 32 + j) = make_float4(
                                 __uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                        if (img) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8)
+                                *reinterpret_cast<uint4*>(img + (b >> 1) * 16384 + swz((uint32_t)v, (uint32_t)((b & 1) * 4 + (j >> 3)))) =
+                                    make_uint4(pack_bf16x2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])),
+                                               pack_bf16x2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])),
+                                               pack_bf16x2(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5])),
+                                               pack_bf16x2(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7])));
+                        }
                     }
                 }
             } else {
@@ -463,7 +501,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 const int c16 = v & 15, r0 = v >> 4;
-                uint16_t* obase = out + ((size_t)t0 * Hv + h) * kD + c16 * 8;
+                uint16_t* obase = out_ptr + ((size_t)t0 * Hv + h) * kD + c16 * 8;
                 const size_t ostride = (size_t)Hv * kD;
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
@@ -493,7 +531,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
 cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                                  const float* initial_state, void* out, float* final_state, uint8_t* ws,
-                                 const WsLayout& L, int num_seqs, int Hqk, int Hv, cudaStream_t st) {
+                                 const WsLayout& L, int num_seqs, int Hqk, int Hv, int segs, cudaStream_t st) {
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(gdn_prefill_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -501,8 +539,8 @@ cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, c
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    gdn_prefill_chain_kernel<<<(unsigned)((long long)num_seqs * Hv), kChainThreads, kChainSmem, st>>>(
-        mq, mk, mv, initial_state, (uint16_t*)out, final_state, ws, L, Hqk, Hv);
+    gdn_prefill_chain_kernel<<<(unsigned)((long long)num_seqs * (2 * segs - 1) * Hv), kChainThreads, kChainSmem, st>>>(
+        mq, mk, mv, initial_state, (uint16_t*)out, final_state, ws, L, Hqk, Hv, segs);
     return cudaGetLastError();
 }
 

@@ -1,11 +1,34 @@
 // Host side of the chunked WY / UT-transform prefill: workspace sizing, TMA tensor maps for
-// the caller's q/k/v tensors, and the three launches (chunk table, intra-chunk, chain).
+// the caller's q/k/v tensors, and the launches (chunk table, intra-chunk, chain, and the scan
+// over runs of chunks when sequences are few and long).
+#include <cstdlib>
+
 #include "gdn_prefill_ws.cuh"
 
 namespace gdn {
 
-size_t prefill_chunked_workspace_bytes(int total_tokens, int num_seqs, int /*Hqk*/, int Hv) {
-    return ws_layout(total_tokens, num_seqs, Hv).total;
+size_t prefill_chunked_workspace_bytes(int total_tokens, int num_seqs, int /*Hqk*/, int Hv, bool allow_split) {
+    return ws_layout(total_tokens, num_seqs, Hv, allow_split).total;
+}
+
+// How many runs of chunks each sequence is cut into: as many as keep every chain CTA resident at
+// once, while a run stays at least kMinSegChunks chunks long.  One run = the plain chain.
+static int choose_segments(const WsLayout& L, int num_seqs, int Hv, int max_seqlen) {
+    if (L.seg_cap <= 1) return 1;
+    static int sms[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+    if (!sms[dev] && cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 1;
+    int segs = seg_cap_for((long long)num_seqs * Hv, sms[dev]);
+    if (segs > L.seg_cap) segs = L.seg_cap;
+    const int by_length = ((max_seqlen + kChunk - 1) / kChunk) / kMinSegChunks;
+    if (segs > by_length) segs = by_length;
+    // GDN_PREFILL_MAX_SEGMENTS (environment, optional) lowers the limit; 1 switches the split off
+    if (const char* env = getenv("GDN_PREFILL_MAX_SEGMENTS")) {
+        const int lim = atoi(env);
+        if (lim >= 1 && segs > lim) segs = lim;
+    }
+    return segs < 1 ? 1 : segs;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -41,10 +64,10 @@ cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v
                                      const float* beta, const float* A_log, const float* dt_bias,
                                      const int32_t* cu_seqlens, const float* initial_state,
                                      void* out, float* final_state, int total_tokens, int num_seqs,
-                                     int /*max_seqlen*/, int Hqk, int Hv, void* workspace, size_t /*workspace_bytes*/,
-                                     cudaStream_t st) {
+                                     int max_seqlen, int Hqk, int Hv, void* workspace, size_t /*workspace_bytes*/,
+                                     bool allow_split, cudaStream_t st) {
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    const WsLayout L = ws_layout(total_tokens, num_seqs, Hv);
+    const WsLayout L = ws_layout(total_tokens, num_seqs, Hv, allow_split);
     cudaError_t e = launch_prefill_prep(cu_seqlens, num_seqs, total_tokens, ws, L, st);
     if (e != cudaSuccess) return e;
     if (total_tokens > 0) {
@@ -54,7 +77,15 @@ cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v
             return cudaErrorUnknown;
         e = launch_prefill_intra(mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv, st);
         if (e != cudaSuccess) return e;
-        e = launch_prefill_chain(mq, mk, mv, initial_state, out, final_state, ws, L, num_seqs, Hqk, Hv, st);
+        const int segs = choose_segments(L, num_seqs, Hv, max_seqlen);
+        e = launch_prefill_chain(mq, mk, mv, initial_state, out, final_state, ws, L, num_seqs, Hqk, Hv, segs, st);
+        if (e != cudaSuccess) return e;
+        if (segs > 1) {
+            CUtensorMap mout, mqt;
+            if (!make_map(&mout, out, total_tokens, Hv) || !make_map(&mqt, ws + L.off_qt, total_tokens, Hv))
+                return cudaErrorUnknown;
+            e = launch_prefill_scan(mout, mqt, out, final_state, ws, L, num_seqs, max_seqlen, Hv, segs, st);
+        }
         if (e != cudaSuccess) return e;
     } else if (final_state) {
         // all sequences are empty: the states pass through

@@ -4,13 +4,13 @@
 #include "gdn_common.cuh"
 
 namespace gdn {
-size_t prefill_chunked_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv);
+size_t prefill_chunked_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv, bool allow_split);
 cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v, const float* g,
                                      const float* beta, const float* A_log, const float* dt_bias,
                                      const int32_t* cu_seqlens, const float* initial_state,
                                      void* out, float* final_state, int total_tokens, int num_seqs,
                                      int max_seqlen, int Hqk, int Hv, void* workspace, size_t workspace_bytes,
-                                     cudaStream_t st);
+                                     bool allow_split, cudaStream_t st);
 }  // namespace gdn
 
 // The scratch itself.  Every device that loads the library carries these bytes until the
@@ -39,7 +39,7 @@ extern "C" int gdn_prefill_static(const void* q, const void* k, const void* v, c
         return GDN_ERR_ALIGN;
     if ((long long)num_seqs * Hv * 16 > 0x7fffffffLL) return GDN_ERR_SHAPE;
     // sizes beyond the fixed scratch are refused, never truncated
-    if (prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv) > (size_t)GDN_PREFILL_STATIC_SCRATCH_BYTES)
+    if (prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv, false) > (size_t)GDN_PREFILL_STATIC_SCRATCH_BYTES)
         return GDN_ERR_WORKSPACE;
 
     int dev = 0;
@@ -57,6 +57,6 @@ extern "C" int gdn_prefill_static(const void* q, const void* k, const void* v, c
     }
     cudaError_t e = prefill_chunked_dispatch(q, k, v, g, beta, nullptr, nullptr, cu_seqlens, initial_state, out, final_state,
                                              total_tokens, num_seqs, max_seqlen, Hqk, Hv, g_static_scratch_addr[dev],
-                                             (size_t)GDN_PREFILL_STATIC_SCRATCH_BYTES, (cudaStream_t)stream);
+                                             (size_t)GDN_PREFILL_STATIC_SCRATCH_BYTES, false, (cudaStream_t)stream);
     return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }

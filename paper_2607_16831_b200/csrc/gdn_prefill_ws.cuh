@@ -13,15 +13,42 @@ constexpr int kABytes = 32768;     // per (chunk, head): T'hi 8K | T'lo 8K | W 1
 constexpr int kPBytes = 8192;      // per (chunk, head): P (swizzled image)
 constexpr int kStatusTimeout = 1;  // device status: a bounded wait ran out
 
+constexpr int kAssumedSMs = 148;   // co-resident chain CTAs the segment split is sized for
+constexpr int kMaxSegments = 8;    // segments a sequence is split into at most
+constexpr int kMinSegChunks = 4;   // a segment is at least this many chunks long
+
 struct WsLayout {
     int nc_max;
-    size_t off_chunk_off, off_seq_order, off_chunk_info, off_scal, off_A, off_P, total;
+    int seg_cap;  // largest number of segments per sequence this workspace has room for (1 = no split)
+    size_t off_chunk_off, off_seq_order, off_chunk_info, off_scal, off_A, off_P, off_qt, off_seg, total;
 };
+
+// Largest S with (sequences x value heads) x (2S - 1) chain CTAs resident at once: segment 0 runs
+// the recurrence itself, every later segment runs it twice (from the zero state and from the
+// identity, see gdn_prefill_scan.cu).
+__host__ __device__ inline int seg_cap_for(long long chains, int sms) {
+    if (chains <= 0) return 1;
+    long long s = (sms / chains + 1) / 2;
+    return (int)(s < 1 ? 1 : (s > kMaxSegments ? kMaxSegments : s));
+}
+
+// Per (sequence, segment >= 1, value head): four 64 KB blocks, three of them fp32 [128][128].
+constexpr int kSegH = 0;       // state reached from the zero state over the segment
+constexpr int kSegP = 1;       // transition: state reached from the identity with v = 0
+constexpr int kSegSin = 2;     // true state entering the segment
+constexpr int kSegSinImg = 3;  // the same in bf16 as two swizzled [128 v][64 k] operand tiles (32 KB used)
+constexpr int kSegBlocks = 4;
+constexpr size_t kSegBlockBytes = (size_t)kD * kD * sizeof(float);
+__host__ __device__ inline size_t seg_block_offset(const WsLayout& L, int n, int s, int h, int Hv, int which) {
+    return L.off_seg + ((((size_t)n * (L.seg_cap - 1) + (s - 1)) * Hv + h) * kSegBlocks + which) * kSegBlockBytes;
+}
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-__host__ __device__ inline WsLayout ws_layout(int total_tokens, int num_seqs, int Hv) {
+__host__ __device__ inline WsLayout ws_layout(int total_tokens, int num_seqs, int Hv, bool allow_split) {
     WsLayout L;
+    L.seg_cap = allow_split ? seg_cap_for((long long)num_seqs * Hv, kAssumedSMs) : 1;
+    if (total_tokens / kChunk < 2 * kMinSegChunks) L.seg_cap = 1;
     L.nc_max = total_tokens / kChunk + num_seqs;  // >= sum over sequences of ceil(len/64)
     size_t o = 1024;                              // header: [0] status, [1] total chunks
     L.off_chunk_off = o;
@@ -36,6 +63,13 @@ __host__ __device__ inline WsLayout ws_layout(int total_tokens, int num_seqs, in
     o += (size_t)L.nc_max * Hv * kABytes;
     L.off_P = o;
     o += (size_t)L.nc_max * Hv * kPBytes;
+    L.off_qt = o;   // bf16 [T][Hv][128]: queries carried back to the segment start
+    L.off_seg = o;
+    if (L.seg_cap > 1) {
+        o = align_up(o + (size_t)total_tokens * Hv * kD * 2, 1024);
+        L.off_seg = o;
+        o += (size_t)num_seqs * (L.seg_cap - 1) * Hv * kSegBlocks * kSegBlockBytes;
+    }
     L.total = o;
     return L;
 }
@@ -53,8 +87,20 @@ cudaError_t launch_prefill_prep(const int32_t* cu_seqlens, int num_seqs, int tot
 cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, const float* g, const float* beta,
                                  const float* A_log, const float* dt_bias, uint8_t* ws, const WsLayout& L, int Hqk,
                                  int Hv, cudaStream_t st);
+// `segs` > 1 splits every sequence into that many runs of chunks (see gdn_prefill_scan.cu).
 cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                                  const float* initial_state, void* out, float* final_state, uint8_t* ws,
-                                 const WsLayout& L, int num_seqs, int Hqk, int Hv, cudaStream_t st);
+                                 const WsLayout& L, int num_seqs, int Hqk, int Hv, int segs, cudaStream_t st);
+cudaError_t launch_prefill_scan(const CUtensorMap& mout, const CUtensorMap& mqt, void* out, float* final_state,
+                                uint8_t* ws, const WsLayout& L, int num_seqs, int max_seqlen, int Hv, int segs,
+                                cudaStream_t st);
+
+// Chunks [first, first + count) of segment `s` when a sequence of `nchunks` chunks is cut into `segs`.
+__host__ __device__ inline void segment_range(int nchunks, int segs, int s, int& first, int& count) {
+    const int m = (nchunks + segs - 1) / segs;
+    first = s * m < nchunks ? s * m : nchunks;
+    const int end = (s + 1) * m < nchunks ? (s + 1) * m : nchunks;
+    count = end - first;
+}
 
 }  // namespace gdn

@@ -69,4 +69,7 @@ def test_workspace_size_grows_with_tokens(gdn):
     a = gdn.gdn_prefill_workspace_bytes(64, 1, 1, 1)
     b = gdn.gdn_prefill_workspace_bytes(4096, 1, 16, 32)
     c = gdn.gdn_prefill_workspace_bytes(4096, 16, 16, 32)
-    assert 0 < a < b <= c
+    d = gdn.gdn_prefill_workspace_bytes(8192, 16, 16, 32)
+    e = gdn.gdn_prefill_workspace_bytes(8192, 1, 16, 32)
+    # few long sequences get extra room for the sequence-parallel scan, so b may exceed c
+    assert 0 < a < b < e and a < c < d

@@ -1,0 +1,93 @@
+"""Sequence-parallel prefill (runs of chunks advanced side by side, joined by the scan over
+chunk-run transitions) against the fp64 CPU oracle, through the C ABI.
+
+The library picks the number of runs from (sequences x value heads) and the longest sequence, so
+the shapes below are what selects 2, 4, 5 and 8 runs; GDN_PREFILL_MAX_SEGMENTS=1 switches the
+split off for the A/B comparison."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from gdn_inputs import config, make_cu_seqlens, make_state, make_tokens
+from paper_2607_16831_b200 import harness
+
+pytestmark = pytest.mark.gpu
+
+
+def custom(lengths, Hqk, Hv, seed, initial=True, **tok_kw):
+    T = int(np.sum(lengths))
+    tok = make_tokens(T, Hqk, Hv, seed=seed, **tok_kw)
+    init = make_state(len(lengths), Hv, seed=seed) if initial else None
+    return dict(kind="prefill", tokens=tok, cu_seqlens=make_cu_seqlens(lengths), initial_state=init, N=len(lengths))
+
+
+def check(cfg, what, **kw):
+    res = harness.run_prefill(cfg, **kw)
+    assert res["device_status"] == 0, "%s: a bounded device wait ran out" % what
+    ref_o, ref_s = oracle.prefill(*harness.token_arrays(cfg["tokens"]), cfg["cu_seqlens"], cfg["initial_state"])
+    e = harness.assert_close(res["out"], ref_o, res["final_state"] if kw.get("want_final", True) else None,
+                             ref_s if kw.get("want_final", True) else None, what)
+    print(what, e)
+    return e, res
+
+
+# (lengths, Hqk, Hv): runs chosen = min((148 / (N Hv) + 1) / 2, 8, chunks / 4)
+SHAPES = [
+    ([512], 4, 8, "8 chunks -> 2 runs"),
+    ([1024], 4, 8, "16 chunks -> 4 runs"),
+    ([2048], 4, 8, "32 chunks -> 8 runs"),
+    ([1000], 4, 8, "ragged tail, 16 chunks -> 4 runs of 4"),
+    ([1217], 2, 4, "20 chunks -> 5 runs, ragged"),
+    ([1100], 8, 16, "18 chunks, 16 heads -> 4 runs (5,5,5,3)"),
+    ([1500, 700], 4, 8, "two sequences -> 5 runs each; the short one has runs of 3, 3, 3, 2, 0 chunks"),
+    ([900, 0, 64], 2, 4, "an empty sequence and a one-chunk sequence beside a split one"),
+]
+
+
+@pytest.mark.parametrize("lengths,Hqk,Hv,what", SHAPES)
+@pytest.mark.parametrize("gate_mean", [2.0, 6.0])
+def test_split_prefill_matches_oracle(lengths, Hqk, Hv, what, gate_mean):
+    # gate_mean 6 (weak decay): the state entering a run matters for all of its tokens
+    check(custom(lengths, Hqk, Hv, seed=len(lengths) * 1000 + lengths[0], gate_mean=gate_mean), what)
+
+
+def test_split_prefill_zero_initial_state_and_no_final_state():
+    cfg = custom([1024], 4, 8, seed=3, initial=False, gate_mean=5.0)
+    check(cfg, "zero initial state, 4 runs")
+    check(cfg, "final state not requested, 4 runs", want_final=False)
+    cfg2 = custom([512], 4, 8, seed=4, gate_mean=5.0)
+    check(cfg2, "final state not requested, 2 runs", want_final=False)
+
+
+def test_split_prefill_full_size_long_sequence():
+    """The T=4096, 16/32-head workload takes the two-run path."""
+    check(config("prefill_long", initial=True, gate_mean=5.0), "prefill_long weak decay, 2 runs")
+
+
+def test_split_and_unsplit_agree():
+    cfg = custom([2048], 4, 8, seed=21, gate_mean=6.0)
+    _, a = check(cfg, "8 runs")
+    os.environ["GDN_PREFILL_MAX_SEGMENTS"] = "1"
+    try:
+        _, b = check(cfg, "1 run")
+    finally:
+        del os.environ["GDN_PREFILL_MAX_SEGMENTS"]
+    assert harness.rel_fro(a["out"], b["out"]) < 8e-3
+    assert harness.rel_fro(a["final_state"], b["final_state"]) < 5e-3
+    # the two paths round differently; identical bits would mean the split was not taken
+    assert not np.array_equal(a["out"], b["out"])
+
+
+def test_split_prefill_correlated_keys():
+    """Keys sharing a common direction: transitions far from a multiple of the identity."""
+    check(custom([1024], 4, 8, seed=23, gate_mean=6.0, key_correlation=0.5), "correlated keys, 4 runs")
+
+
+def test_split_prefill_repeated_calls_reuse_workspace():
+    cfg = custom([1024], 4, 8, seed=29, gate_mean=4.0)
+    _, a = check(cfg, "first call")
+    _, b = check(cfg, "second call")
+    np.testing.assert_array_equal(a["out"], b["out"])
+    np.testing.assert_array_equal(a["final_state"], b["final_state"])
