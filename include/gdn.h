@@ -137,6 +137,13 @@ size_t gdn_prefill_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int 
  * differently.
  * The number of runs follows from num_seqs, Hv and max_seqlen; the environment variable
  * GDN_PREFILL_MAX_SEGMENTS (1..8) lowers it, 1 switches the split off.
+ *
+ * At the other end, when max_seqlen <= 64 (no sequence longer than one chunk) and a cost model
+ * fitted to measurements says the token-serial kernel of gdn_prefill_recurrent is faster (a few
+ * short sequences, or many sequences of a handful of tokens), gdn_prefill runs that kernel
+ * instead: the narrow short-shape fallback beside a chunked main path that Sections 5.3 and
+ * 5.5 mention.  GDN_PREFILL_SHORT_FALLBACK=0 in the environment keeps the chunked kernels.
+ * The workspace is required (and checked) either way.
  */
 int gdn_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
                 const int32_t* cu_seqlens, const float* initial_state, void* out, float* final_state,

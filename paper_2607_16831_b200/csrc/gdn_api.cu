@@ -1,4 +1,5 @@
 // C-ABI entry points of libgdn: argument validation and launch dispatch only.
+#include <cstdlib>
 #include <stdio.h>
 #include <stdlib.h>
 
@@ -96,6 +97,23 @@ static int check_prefill(const void* q, const void* k, const void* v, const floa
     return GDN_OK;
 }
 
+// Short-sequence dispatch of gdn_prefill.  When no sequence is longer than one chunk the chunked
+// path pays for whole 64-token chunks and three dependent launches (about 27 us even for a few
+// tokens), while the token-serial kernel costs about 0.6 us per token of the longest sequence,
+// times the number of waves its (sequence, head) units need.  Both models are fits to
+// measurements on B200 over 1..64 sequences of 4..128 tokens at 8 and 32 value heads; the faster
+// one by the model is used.  GDN_PREFILL_SHORT_FALLBACK=0 (environment) keeps the chunked path.
+static bool prefer_token_serial(int num_seqs, int Hv, int max_seqlen) {
+    if (max_seqlen > kChunk) return false;
+    if (const char* env = getenv("GDN_PREFILL_SHORT_FALLBACK"))
+        if (env[0] == '0') return false;
+    const double chains = (double)num_seqs * Hv;
+    const double waves = chains > 96.0 ? chains / 96.0 : 1.0;
+    const double t_serial = 2.0 + 0.014 * chains + 0.6 * max_seqlen * waves;
+    const double t_chunked = 0.098 * chains > 27.0 ? 0.098 * chains : 27.0;
+    return t_serial < t_chunked;
+}
+
 }  // namespace gdn
 
 using namespace gdn;
@@ -167,6 +185,13 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
     const size_t need = prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv, true);
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
         return GDN_ERR_WORKSPACE;
+    if (prefer_token_serial(num_seqs, Hv, max_seqlen)) {
+        // the device status word the chunked kernels would have cleared
+        cudaMemsetAsync(workspace, 0, 8, (cudaStream_t)stream);
+        return cuda_status(prefill_recurrent_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
+                                                      total_tokens, num_seqs, Hqk, Hv, (cudaStream_t)stream),
+                           "gdn_prefill (token-serial)");
+    }
     return cuda_status(prefill_chunked_dispatch(q, k, v, g, beta, nullptr, nullptr, cu_seqlens, initial_state, out,
                                                 final_state, total_tokens, num_seqs, max_seqlen, Hqk, Hv, workspace,
                                                 workspace_bytes, true, (cudaStream_t)stream), "gdn_prefill");

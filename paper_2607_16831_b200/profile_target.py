@@ -20,6 +20,8 @@ def main():
     ap.add_argument("--workload", default="decode", choices=["decode", "prefill_long", "prefill_varlen", "prefill_tiny"])
     ap.add_argument("--B", type=int, default=64)
     ap.add_argument("--T", type=int, default=4096)
+    ap.add_argument("--Hqk", type=int, default=16)
+    ap.add_argument("--Hv", type=int, default=32)
     ap.add_argument("--calls", type=int, default=3)
     ap.add_argument("--initial", action="store_true")
     ap.add_argument("--recurrent", action="store_true")
@@ -46,7 +48,7 @@ def main():
             ev[i][1].record()
     else:
         over = {"T": args.T, "initial": args.initial} if args.workload == "prefill_long" else {}
-        cfg = config(args.workload, **over)
+        cfg = config(args.workload, Hqk=args.Hqk, Hv=args.Hv, **over)
         tok = cfg["tokens"]
         d = harness.to_device(tok)
         cu_np = np.asarray(cfg["cu_seqlens"], dtype=np.int32)

@@ -9,6 +9,13 @@ from paper_2607_16831_b200 import harness
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(autouse=True)
+def chunked_path_only(monkeypatch):
+    """These tests are about the chunked kernels: keep gdn_prefill from handing the shortest
+    shapes to the token-serial kernel (tests/test_prefill_dispatch_gpu.py covers that hand-over)."""
+    monkeypatch.setenv("GDN_PREFILL_SHORT_FALLBACK", "0")
+
+
 def check(cfg, what, **kw):
     res = harness.run_prefill(cfg, **kw)
     assert res["device_status"] == 0, "%s: a bounded device wait ran out" % what
