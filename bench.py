@@ -181,14 +181,25 @@ def decode_buffers(B, seed=0, min_footprint=600e6):
     return cfg, d, s_in, s_out, out, nbuf
 
 
-def bench_prefill(name, peaks, reps, **over):
-    """Whole-call device time of gdn_prefill (prep + intra-chunk + chain kernels)."""
+def bench_prefill(name, peaks, reps, env=None, lengths=None, **over):
+    """Whole-call device time of gdn_prefill (chunk table + intra-chunk + chain kernels, plus the
+    scan over runs of chunks when the library splits long sequences).  `env` holds library
+    switches set for the duration of this measurement; `lengths` replaces the workload's
+    sequence lengths (same token recipe)."""
     import torch
     import paper_2607_16831_b200 as gdn
     from gdn_inputs import config
     from paper_2607_16831_b200 import harness
 
-    cfg = config(name, **over)
+    saved = {k: os.environ.get(k) for k in (env or {})}
+    os.environ.update(env or {})
+    if lengths is None:
+        cfg = config(name, **over)
+    else:
+        from gdn_inputs import make_cu_seqlens, make_state, make_tokens
+        Hqk, Hv = over.get("Hqk", 16), over.get("Hv", 32)
+        cfg = dict(tokens=make_tokens(int(np.sum(lengths)), Hqk, Hv, seed=0), cu_seqlens=make_cu_seqlens(lengths),
+                   initial_state=make_state(len(lengths), Hv, seed=0))
     tok = cfg["tokens"]
     d = harness.to_device(tok)
     cu_np = np.asarray(cfg["cu_seqlens"], dtype=np.int32)
@@ -219,11 +230,17 @@ def bench_prefill(name, peaks, reps, **over):
         torch.cuda.synchronize()
         ts.append(a.elapsed_time(b) * 1e-3)
     t = float(np.median(ts))
+    for k, v in saved.items():
+        if v is None:
+            del os.environ[k]
+        else:
+            os.environ[k] = v
     nstate = (1 if init is not None else 0) + 1
     alg_bytes = tok.T * PREFILL_BYTES_PER_TOKEN * (tok.Hv / 32.0) + nstate * N * tok.Hv * 65536
     flops = tok.T * PREFILL_FLOPS_PER_TOKEN * (tok.Hv / 32.0)
     return {
-        "workload": name, "tokens": int(tok.T), "num_seqs": int(N), "us": t * 1e6, "tokens_per_s": tok.T / t,
+        "workload": name, "tokens": int(tok.T), "num_seqs": int(N), "heads": "%d/%d" % (tok.Hqk, tok.Hv),
+        "us": t * 1e6, "tokens_per_s": tok.T / t,
         "hbm": {"achieved_gbs": alg_bytes / t / 1e9, "frac": alg_bytes / t / 1e9 / peaks["hbm"]},
         "tensor": {"achieved_tflops": flops / t / 1e12, "frac": flops / t / 1e12 / peaks["bf16"]},
         "chain_steps": int(np.max((np.diff(cu_np) + 63) // 64)),
@@ -416,6 +433,18 @@ def run_gpu(args):
         pre.append(dict(bench_prefill("prefill_long", peaks, reps), variant="zero initial state"))
         pre.append(dict(bench_prefill("prefill_long", peaks, reps, initial=True), variant="N(0,0.02) initial state"))
         pre.append(dict(bench_prefill("prefill_varlen", peaks, reps), variant="16 sequences U[1,2048]"))
+        pre.append(dict(bench_prefill("prefill_long", peaks, reps, env={"GDN_PREFILL_MAX_SEGMENTS": "1"}),
+                        variant="zero initial state, sequence split switched off (one chain CTA per head)"))
+        # smaller head counts (4 key / 8 value heads), where one sequence leaves even more of the GPU idle
+        pre.append(dict(bench_prefill("prefill_long", peaks, reps, Hqk=4, Hv=8), variant="4/8 heads, 8 runs of chunks"))
+        pre.append(dict(bench_prefill("prefill_long", peaks, reps, Hqk=4, Hv=8, env={"GDN_PREFILL_MAX_SEGMENTS": "1"}),
+                        variant="4/8 heads, sequence split switched off"))
+        pre.append(dict(bench_prefill("prefill_varlen", peaks, reps, Hqk=4, Hv=8), variant="4/8 heads, 16 sequences U[1,2048]"))
+        pre.append(dict(bench_prefill("short", peaks, reps, lengths=[8] * 64, Hqk=4, Hv=8),
+                        variant="4/8 heads, 64 sequences of 8 tokens (token-serial kernel chosen)"))
+        pre.append(dict(bench_prefill("short", peaks, reps, lengths=[8] * 64, Hqk=4, Hv=8,
+                                      env={"GDN_PREFILL_SHORT_FALLBACK": "0"}),
+                        variant="4/8 heads, 64 sequences of 8 tokens, chunked kernels forced"))
         line["prefill"] = {"rooflines": {"hbm_gbs": peaks["hbm"], "bf16_tflops": peaks["bf16"], "source": peaks["source"],
                                          "bytes_per_token": PREFILL_BYTES_PER_TOKEN,
                                          "flops_per_token": PREFILL_FLOPS_PER_TOKEN}, "runs": pre}
