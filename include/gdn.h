@@ -216,6 +216,44 @@ int gdn_prefill_static(const void* q, const void* k, const void* v, const float*
                        int Hqk, int Hv, int dk, int dv, void* stream);
 
 /*
+ * Building blocks of sequence-parallel prefill: one long sequence (or each of several) cut into
+ * consecutive pieces that are processed at the same time, e.g. one piece per GPU.  The paper
+ * evaluates single-GPU kernels only and has no counterpart; the algebra is the recurrence of
+ * Section 3.2 written as an affine map of the state.  Over a piece of tokens, with M_t the
+ * product of the per-token transitions alpha (I - beta k k^T) from the start of the piece up to
+ * token t and H_t the state reached from the zero state,
+ *
+ *     S_t = S_in M_t + H_t,        o_t = S_t q_t = H_t q_t + S_in (M_t q_t).
+ *
+ * gdn_prefill_partial   runs a piece without knowing S_in.  Arguments as gdn_prefill, and
+ *     out0  bf16 [T_tot, Hv, dv]       H_t q_t (the outputs the zero state would give)
+ *     qt    bf16 [T_tot, Hv, dk]       M_t q_t (queries carried back to the start of the piece)
+ *     H     fp32 [num_seqs, Hv, dv, dk]   H at the end of each sequence of the piece
+ *     P     fp32 [num_seqs, Hv, dk, dk]   M at the end: S_end = S_in P + H
+ *     workspace: as gdn_prefill.  An empty sequence gives H = 0, P = I.
+ * gdn_state_scan        folds pieces in order: S_out = (...((S0 P_0 + H_0) P_1 + H_1)...), fp32.
+ *     P, H  fp32 [steps, num_seqs, Hv, 128, 128] (for instance the all-gathered results of the
+ *           pieces before this one); S0 fp32 [num_seqs, Hv, dv, dk] or NULL (zeros);
+ *           S_out may alias S0 exactly.  steps = 0 copies S0.
+ * gdn_prefill_apply     finishes a piece once its entering state is known:
+ *     out[t] += S_in qt[t] for every token (out holds out0 on entry; rounded to bf16 again).
+ *     S_in fp32 [num_seqs, Hv, dv, dk]; workspace >= 1024 + num_seqs * Hv * 32768 bytes,
+ *     1024-byte aligned (a gdn_prefill workspace for the same sizes is large enough).
+ * The state leaving a piece is gdn_state_scan(S_in, P, H, steps = 1).
+ * A piece that starts a sequence can instead run gdn_prefill with the known initial state and
+ * publish (P, H) = (0, its final state).
+ */
+int gdn_prefill_partial(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                        const int32_t* cu_seqlens, void* out0, void* qt, float* H, float* P,
+                        int total_tokens, int num_seqs, int max_seqlen, int Hqk, int Hv, int dk, int dv,
+                        void* workspace, size_t workspace_bytes, void* stream);
+int gdn_state_scan(const float* S0, const float* P, const float* H, int steps, float* S_out,
+                   int num_seqs, int Hv, int dk, int dv, void* stream);
+int gdn_prefill_apply(const float* S_in, const void* qt, void* out, const int32_t* cu_seqlens,
+                      int total_tokens, int num_seqs, int max_seqlen, int Hv, int dk, int dv,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Reads (and clears) the device-side status word that the prefill kernels set when a
  * bounded wait on an asynchronous copy or tensor-core completion ran out.  HOST
  * pointer out; synchronises `stream`.  *device_status == 0 means no kernel gave up.

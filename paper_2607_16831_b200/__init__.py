@@ -21,6 +21,7 @@ STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL", 2: "GDN_ERR_SHAPE", 3: "GDN_ERR_
 EXPORTS = ("gdn_status_string", "gdn_decode", "gdn_decode_variant", "gdn_decode_num_variants",
            "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_recurrent", "gdn_prefill_static",
            "gdn_decode_gated", "gdn_prefill_gated", "gdn_decode_multi",
+           "gdn_prefill_partial", "gdn_state_scan", "gdn_prefill_apply",
            "gdn_last_device_status")
 
 
@@ -64,6 +65,12 @@ def lib() -> ctypes.CDLL:
         L.gdn_decode_gated.restype = I
         L.gdn_prefill_gated.argtypes = [P] * 11 + [I] * 7 + [P, Z, P]
         L.gdn_prefill_gated.restype = I
+        L.gdn_prefill_partial.argtypes = [P] * 10 + [I] * 7 + [P, Z, P]
+        L.gdn_prefill_partial.restype = I
+        L.gdn_state_scan.argtypes = [P, P, P, I, P, I, I, I, I, P]
+        L.gdn_state_scan.restype = I
+        L.gdn_prefill_apply.argtypes = [P] * 4 + [I] * 6 + [P, Z, P]
+        L.gdn_prefill_apply.restype = I
         L.gdn_last_device_status.argtypes = [P, ctypes.POINTER(I), P]
         L.gdn_last_device_status.restype = I
         _lib = L
@@ -138,6 +145,38 @@ def gdn_prefill_recurrent(q, k, v, g, beta, cu_seqlens, initial_state, out, fina
                                      _ptr(initial_state), _ptr(out), _ptr(final_state), T, N, int(max_seqlen),
                                      Hqk, Hv, dk, dv, _stream(stream))
     _check(rc, "gdn_prefill_recurrent")
+
+
+def gdn_prefill_partial(q, k, v, g, beta, cu_seqlens, out0, qt, H, P, max_seqlen: int, workspace, stream=None) -> None:
+    """A piece of every sequence without its entering state: out0 = H_t q_t, qt = M_t q_t (bf16
+    [T,Hv,128]); H, P fp32 [N,Hv,128,128] with S_end = S_in P + H."""
+    T, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    N = cu_seqlens.shape[0] - 1
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().gdn_prefill_partial(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(cu_seqlens), _ptr(out0),
+                                   _ptr(qt), _ptr(H), _ptr(P), T, N, int(max_seqlen), Hqk, Hv, dk, dv,
+                                   _ptr(workspace), wbytes, _stream(stream))
+    _check(rc, "gdn_prefill_partial")
+
+
+def gdn_state_scan(S0, P, H, S_out, stream=None) -> None:
+    """S_out = (...((S0 P[0] + H[0]) P[1] + H[1])...); P, H fp32 [steps,N,Hv,128,128]; S0 fp32
+    [N,Hv,128,128] or None (zeros)."""
+    steps = 0 if P is None else int(P.shape[0])
+    N, Hv, dv, dk = S_out.shape
+    rc = lib().gdn_state_scan(_ptr(S0), _ptr(P), _ptr(H), steps, _ptr(S_out), N, Hv, dk, dv, _stream(stream))
+    _check(rc, "gdn_state_scan")
+
+
+def gdn_prefill_apply(S_in, qt, out, cu_seqlens, max_seqlen: int, workspace, stream=None) -> None:
+    """out[t] += S_in qt[t] for every token of every sequence (out holds gdn_prefill_partial's out0)."""
+    T, Hv, dk = qt.shape
+    N = cu_seqlens.shape[0] - 1
+    wbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().gdn_prefill_apply(_ptr(S_in), _ptr(qt), _ptr(out), _ptr(cu_seqlens), T, N, int(max_seqlen), Hv, dk,
+                                 out.shape[2], _ptr(workspace), wbytes, _stream(stream))
+    _check(rc, "gdn_prefill_apply")
 
 
 def gdn_decode_multi(q, k, v, g, beta, state_in, state_out, out, stream=None) -> None:

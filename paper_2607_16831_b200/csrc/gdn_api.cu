@@ -17,6 +17,15 @@ cudaError_t prefill_recurrent_dispatch(const void* q, const void* k, const void*
                                        void* out, float* final_state, int total_tokens, int num_seqs, int Hqk,
                                        int Hv, cudaStream_t st);
 size_t prefill_chunked_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv, bool allow_split);
+cudaError_t prefill_partial_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                                     const int32_t* cu_seqlens, void* out0, void* qt, float* H, float* P,
+                                     int total_tokens, int num_seqs, int Hqk, int Hv, void* workspace,
+                                     cudaStream_t st);
+cudaError_t prefill_apply_dispatch(const float* S_in, const void* qt, void* out, const int32_t* cu_seqlens,
+                                   int total_tokens, int num_seqs, int max_seqlen, int Hv, void* workspace,
+                                   cudaStream_t st);
+cudaError_t launch_state_scan(const float* S0, const float* P, const float* H, int steps, float* S_out, int num_seqs,
+                              int Hv, cudaStream_t st);
 cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v, const float* g,
                                      const float* beta, const float* A_log, const float* dt_bias,
                                      const int32_t* cu_seqlens, const float* initial_state,
@@ -235,6 +244,57 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const flo
     return cuda_status(prefill_recurrent_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
                                                   total_tokens, num_seqs, Hqk, Hv, (cudaStream_t)stream),
                        "gdn_prefill_recurrent");
+}
+
+int gdn_prefill_partial(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                        const int32_t* cu_seqlens, void* out0, void* qt, float* H, float* P, int total_tokens,
+                        int num_seqs, int max_seqlen, int Hqk, int Hv, int dk, int dv, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    bool nothing = false;
+    if (int rc = check_prefill(q, k, v, g, beta, cu_seqlens, nullptr, out0, nullptr, total_tokens, num_seqs,
+                               max_seqlen, Hqk, Hv, dk, dv, &nothing))
+        return rc;
+    if (nothing) return GDN_OK;
+    if (!H || !P || (total_tokens > 0 && !qt)) return GDN_ERR_NULL;
+    if (!aligned16(H) || !aligned16(P) || !aligned16(qt)) return GDN_ERR_ALIGN;
+    const size_t need = prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv, true);
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
+        return GDN_ERR_WORKSPACE;
+    return cuda_status(prefill_partial_dispatch(q, k, v, g, beta, cu_seqlens, out0, qt, H, P, total_tokens, num_seqs,
+                                                Hqk, Hv, workspace, (cudaStream_t)stream), "gdn_prefill_partial");
+}
+
+int gdn_state_scan(const float* S0, const float* P, const float* H, int steps, float* S_out, int num_seqs, int Hv,
+                   int dk, int dv, void* stream) {
+    if (steps < 0 || num_seqs < 0) return GDN_ERR_SHAPE;
+    if (int rc = check_heads(Hv, Hv, dk, dv)) return rc;
+    if (num_seqs == 0) return GDN_OK;
+    if (!S_out || (steps > 0 && (!P || !H))) return GDN_ERR_NULL;
+    if (!aligned16(S0) || !aligned16(P) || !aligned16(H) || !aligned16(S_out)) return GDN_ERR_ALIGN;
+    if ((long long)num_seqs * Hv > 0x7fffffffLL / 16) return GDN_ERR_SHAPE;
+    if (!device_supported()) return GDN_ERR_UNSUPPORTED;
+    return cuda_status(launch_state_scan(S0, P, H, steps, S_out, num_seqs, Hv, (cudaStream_t)stream), "gdn_state_scan");
+}
+
+int gdn_prefill_apply(const float* S_in, const void* qt, void* out, const int32_t* cu_seqlens, int total_tokens,
+                      int num_seqs, int max_seqlen, int Hv, int dk, int dv, void* workspace, size_t workspace_bytes,
+                      void* stream) {
+    if (total_tokens < 0 || num_seqs < 0 || max_seqlen < 0) return GDN_ERR_SHAPE;
+    if (int rc = check_heads(Hv, Hv, dk, dv)) return rc;
+    if (max_seqlen > total_tokens) return GDN_ERR_SHAPE;
+    if (total_tokens > 0 && (num_seqs == 0 || max_seqlen == 0)) return GDN_ERR_SHAPE;
+    if ((long long)max_seqlen * num_seqs < total_tokens) return GDN_ERR_SHAPE;
+    if (num_seqs == 0 || total_tokens == 0) return GDN_OK;
+    if (!S_in || !qt || !out || !cu_seqlens) return GDN_ERR_NULL;
+    if (!aligned16(S_in) || !aligned16(qt) || !aligned16(out) || (reinterpret_cast<uintptr_t>(cu_seqlens) & 3u))
+        return GDN_ERR_ALIGN;
+    if (num_seqs > 65535) return GDN_ERR_SHAPE;
+    if (!device_supported()) return GDN_ERR_UNSUPPORTED;
+    const size_t need = 1024 + (size_t)num_seqs * Hv * 32768;
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
+        return GDN_ERR_WORKSPACE;
+    return cuda_status(prefill_apply_dispatch(S_in, qt, out, cu_seqlens, total_tokens, num_seqs, max_seqlen, Hv,
+                                              workspace, (cudaStream_t)stream), "gdn_prefill_apply");
 }
 
 int gdn_last_device_status(void* workspace, int* device_status, void* stream) {

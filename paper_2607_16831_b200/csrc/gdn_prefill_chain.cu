@@ -76,13 +76,17 @@ __global__ void __launch_bounds__(kChainThreads, 1)
 gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const __grid_constant__ CUtensorMap map_v, const float* initial_state,
                          uint16_t* __restrict__ out, float* final_state, uint8_t* __restrict__ ws, WsLayout L,
-                         int Hqk, int Hv, int segs) {
-    // CTAs are handed out longest sequence first; within a sequence: run 0, then (zero, identity) per run
-    const int per_seq = 2 * segs - 1;
+                         int Hqk, int Hv, int segs, ChainPartial part) {
+    // CTAs are handed out longest sequence first; within a sequence: run 0, then (zero, identity) per run.
+    // Partial mode (part.H set, segs = 1): every sequence is one run that is walked from the zero state
+    // and from the identity, results to the caller's H, P and qt.
+    const bool partial = part.H != nullptr;
+    const int per_seq = partial ? 2 : 2 * segs - 1;
     const int h = blockIdx.x % Hv, unit = blockIdx.x / Hv;
     const int n = reinterpret_cast<const int*>(ws + L.off_seq_order)[unit / per_seq];
-    const int seg = (unit % per_seq + 1) >> 1;
-    const bool ident = seg > 0 && ((unit % per_seq) & 1) == 0;  // identity start, v = 0
+    const int seg = partial ? 0 : (unit % per_seq + 1) >> 1;
+    const bool ident = partial ? (unit % per_seq) == 1
+                               : (seg > 0 && ((unit % per_seq) & 1) == 0);  // identity start, v = 0
     const int hq = h / (Hv / Hqk);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -99,7 +103,13 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int c_begin = chunk_off[n] + seg_first, c_end = c_begin + nchunks;
 
     if (nchunks <= 0) {  // empty sequence: the state passes through; empty run: nothing to do
-        if (seg == 0 && final_state && tid < kD) {
+        if (partial && tid < kD) {  // H = 0, P = I
+            float* dst = (ident ? part.P : part.H) + ((size_t)n * Hv + h) * kD * kD + (size_t)tid * kD;
+            for (int j = 0; j < kD; j += 4)
+                *reinterpret_cast<float4*>(dst + j) =
+                    make_float4((ident && tid == j) ? 1.f : 0.f, (ident && tid == j + 1) ? 1.f : 0.f,
+                                (ident && tid == j + 2) ? 1.f : 0.f, (ident && tid == j + 3) ? 1.f : 0.f);
+        } else if (seg == 0 && final_state && tid < kD) {
             const size_t sb0 = ((size_t)n * Hv + h) * kD * kD + (size_t)tid * kD;
             for (int j = 0; j < kD; j += 4) {
                 float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -114,12 +124,14 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int t_end = chunk_info[c_end - 1].y + chunk_info[c_end - 1].z;
     // where this CTA's state comes from and where its results go
     const size_t state_off = ((size_t)n * Hv + h) * kD * kD;
-    const float* init_ptr = (seg == 0 && initial_state) ? initial_state + state_off : nullptr;
+    const float* init_ptr = (!partial && seg == 0 && initial_state) ? initial_state + state_off : nullptr;
     float* fin_ptr = final_state ? final_state + state_off : nullptr;
-    if (segs > 1)
+    if (partial)
+        fin_ptr = (ident ? part.P : part.H) + state_off;
+    else if (segs > 1)
         fin_ptr = reinterpret_cast<float*>(
             ws + seg_block_offset(L, n, seg == 0 ? 1 : seg, h, Hv, seg == 0 ? kSegSin : (ident ? kSegP : kSegH)));
-    uint16_t* out_ptr = ident ? reinterpret_cast<uint16_t*>(ws + L.off_qt) : out;
+    uint16_t* out_ptr = ident ? (partial ? part.qt : reinterpret_cast<uint16_t*>(ws + L.off_qt)) : out;
 
     if (tid == 0) {
         for (int i = 0; i < B_COUNT; ++i) {
@@ -531,7 +543,8 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
 cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                                  const float* initial_state, void* out, float* final_state, uint8_t* ws,
-                                 const WsLayout& L, int num_seqs, int Hqk, int Hv, int segs, cudaStream_t st) {
+                                 const WsLayout& L, int num_seqs, int Hqk, int Hv, int segs, const ChainPartial& part,
+                                 cudaStream_t st) {
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(gdn_prefill_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -539,8 +552,9 @@ cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, c
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    gdn_prefill_chain_kernel<<<(unsigned)((long long)num_seqs * (2 * segs - 1) * Hv), kChainThreads, kChainSmem, st>>>(
-        mq, mk, mv, initial_state, (uint16_t*)out, final_state, ws, L, Hqk, Hv, segs);
+    const int per_seq = part.H ? 2 : 2 * segs - 1;
+    gdn_prefill_chain_kernel<<<(unsigned)((long long)num_seqs * per_seq * Hv), kChainThreads, kChainSmem, st>>>(
+        mq, mk, mv, initial_state, (uint16_t*)out, final_state, ws, L, Hqk, Hv, segs, part);
     return cudaGetLastError();
 }
 

@@ -2,6 +2,7 @@
 // the caller's q/k/v tensors, and the launches (chunk table, intra-chunk, chain, and the scan
 // over runs of chunks when sequences are few and long).
 #include <cstdlib>
+#include <cstring>
 
 #include "gdn_prefill_ws.cuh"
 
@@ -78,7 +79,8 @@ cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v
         e = launch_prefill_intra(mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv, st);
         if (e != cudaSuccess) return e;
         const int segs = choose_segments(L, num_seqs, Hv, max_seqlen);
-        e = launch_prefill_chain(mq, mk, mv, initial_state, out, final_state, ws, L, num_seqs, Hqk, Hv, segs, st);
+        e = launch_prefill_chain(mq, mk, mv, initial_state, out, final_state, ws, L, num_seqs, Hqk, Hv, segs,
+                                 ChainPartial{nullptr, nullptr, nullptr}, st);
         if (e != cudaSuccess) return e;
         if (segs > 1) {
             CUtensorMap mout, mqt;
@@ -98,6 +100,42 @@ cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v
         }
     }
     return cudaGetLastError();
+}
+
+// One run of every sequence walked from the zero state and from the identity (see gdn_prefill_scan.cu).
+cudaError_t prefill_partial_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                                     const int32_t* cu_seqlens, void* out0, void* qt, float* H, float* P,
+                                     int total_tokens, int num_seqs, int Hqk, int Hv, void* workspace,
+                                     cudaStream_t st) {
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const WsLayout L = ws_layout(total_tokens, num_seqs, Hv, false);
+    cudaError_t e = launch_prefill_prep(cu_seqlens, num_seqs, total_tokens, ws, L, st);
+    if (e != cudaSuccess) return e;
+    CUtensorMap mq, mk, mv;
+    if (total_tokens > 0) {
+        if (!make_map(&mq, q, total_tokens, Hqk) || !make_map(&mk, k, total_tokens, Hqk) ||
+            !make_map(&mv, v, total_tokens, Hv))
+            return cudaErrorUnknown;
+        e = launch_prefill_intra(mq, mk, g, beta, nullptr, nullptr, ws, L, Hqk, Hv, st);
+        if (e != cudaSuccess) return e;
+    } else {
+        // no tensor to describe; every sequence is empty and the chain CTAs return before using the maps
+        memset(&mq, 0, sizeof mq);
+        mk = mq;
+        mv = mq;
+    }
+    return launch_prefill_chain(mq, mk, mv, nullptr, out0, nullptr, ws, L, num_seqs, Hqk, Hv, 1,
+                                ChainPartial{H, P, static_cast<uint16_t*>(qt)}, st);
+}
+
+cudaError_t prefill_apply_dispatch(const float* S_in, const void* qt, void* out, const int32_t* cu_seqlens,
+                                   int total_tokens, int num_seqs, int max_seqlen, int Hv, void* workspace,
+                                   cudaStream_t st) {
+    if (total_tokens == 0) return cudaSuccess;
+    CUtensorMap mout, mqt;
+    if (!make_map(&mout, out, total_tokens, Hv) || !make_map(&mqt, qt, total_tokens, Hv)) return cudaErrorUnknown;
+    return launch_prefill_apply(mout, mqt, S_in, out, cu_seqlens, num_seqs, max_seqlen, Hv,
+                                static_cast<uint8_t*>(workspace), st);
 }
 
 }  // namespace gdn

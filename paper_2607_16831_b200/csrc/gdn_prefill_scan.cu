@@ -27,16 +27,33 @@ constexpr uint32_t CB_P = 8192 + 128;  // one or two buffers of P, fp32 [128][12
 constexpr uint32_t kPBlock = (uint32_t)kSegBlockBytes;
 __host__ __device__ constexpr uint32_t combine_smem(int nbuf) { return CB_P + nbuf * kPBlock + 128; }
 
-// grid (sequences x value heads, 128 / 16 row blocks).  `nbuf` = 2 fetches the next run's P while
-// this run's product is computed.
+// Where the scan S <- S P_i + H_i (i = 0 .. steps-1) finds and leaves its operands.  Offsets are in
+// floats from the base pointers: block of (step i, sequence n, head h) = i * ss + n * sn + h * sh.
+struct ScanArgs {
+    const float* x0;        // starting state of (n, h) at n * x_sn + h * x_sh; NULL = zeros
+    long long x_sn, x_sh;
+    const float* P;         // fp32 [128][128] per (i, n, h)
+    const float* H;
+    long long ss, sn, sh;
+    float* sin;             // optional: the state entering step i >= 1 is written to block (i, n, h) ...
+    uint8_t* img;           // ... and as bf16 operand tiles (same block index, 4 bytes per float)
+    float* fin;             // optional: the last state, [N][Hv][128][128]
+    int steps;
+    const int* chunk_off;   // optional: step i is run i + 1 of `segs` runs; stop at the first empty run
+    int segs;
+    int* status;            // device status word
+};
+
+// grid (sequences x value heads, 128 / 16 row blocks).  `nbuf` = 2 fetches the next step's P while
+// this step's product is computed.
 __global__ void __launch_bounds__(128)
-gdn_prefill_combine_kernel(float* final_state, uint8_t* __restrict__ ws, WsLayout L, int Hv, int segs, int nbuf) {
+gdn_prefill_combine_kernel(ScanArgs A, int Hv, int nbuf) {
     const int n = blockIdx.x / Hv, h = blockIdx.x % Hv;
     const int row0 = blockIdx.y * kCombineRows;
     const int tid = threadIdx.x, ty = tid >> 5, tx = tid & 31;  // thread tile: rows 4 ty.., columns 4 tx..
-    const int* chunk_off = reinterpret_cast<const int*>(ws + L.off_chunk_off);
-    const int nch = chunk_off[n + 1] - chunk_off[n];
+    const int nch = A.chunk_off ? A.chunk_off[n + 1] - A.chunk_off[n] : 1;
     if (nch <= 0) return;  // empty sequence: the chain kernel passed the state through
+    const long long unit = (long long)n * A.sn + (long long)h * A.sh;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -45,15 +62,19 @@ gdn_prefill_combine_kernel(float* final_state, uint8_t* __restrict__ ws, WsLayou
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + CB_BAR + 16);
     const float* pbuf = reinterpret_cast<const float*>(smem + CB_P);
 
+    // below, s = i + 1 counts steps from 1 (= the run index when the steps are runs of chunks)
+    const int segs = A.steps + 1;
     auto run_chunks = [&](int s) {
+        if (s >= segs) return 0;
+        if (!A.chunk_off) return 1;
         int first, count;
-        segment_range(nch, segs, s, first, count);
-        return s < segs ? count : 0;
+        segment_range(nch, A.segs, s, first, count);
+        return count;
     };
     auto fetch_P = [&](int s) {  // one thread: the whole 64 KB block in one bulk copy
         const int b = (s - 1) % nbuf;
         mbar_expect_tx(bars + b, kPBlock);
-        bulk_load(smem + CB_P + b * kPBlock, ws + seg_block_offset(L, n, s, h, Hv, kSegP), kPBlock, bars + b);
+        bulk_load(smem + CB_P + b * kPBlock, A.P + (long long)(s - 1) * A.ss + unit, kPBlock, bars + b);
     };
     if (tid == 0) {
         mbar_init(bars + 0, 1);
@@ -65,19 +86,20 @@ gdn_prefill_combine_kernel(float* final_state, uint8_t* __restrict__ ws, WsLayou
 
     float acc[4][4];
     {
-        const float* sin1 = reinterpret_cast<const float*>(ws + seg_block_offset(L, n, 1, h, Hv, kSegSin));
+        const float* x0 = A.x0 ? A.x0 + (long long)n * A.x_sn + (long long)h * A.x_sh : nullptr;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float4 x = *reinterpret_cast<const float4*>(sin1 + (size_t)(row0 + ty * 4 + i) * kD + tx * 4);
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (x0) x = *reinterpret_cast<const float4*>(x0 + (size_t)(row0 + ty * 4 + i) * kD + tx * 4);
             acc[i][0] = x.x; acc[i][1] = x.y; acc[i][2] = x.z; acc[i][3] = x.w;
         }
     }
     for (int s = 1; s < segs; ++s) {
         if (run_chunks(s) <= 0) break;  // later runs are empty as well
-        if (s >= 2) {
+        if (s >= 2 && A.sin) {
             // the state entering run s, for the fix-up: fp32 and as bf16 operand tiles
-            float* sin = reinterpret_cast<float*>(ws + seg_block_offset(L, n, s, h, Hv, kSegSin));
-            uint8_t* img = ws + seg_block_offset(L, n, s, h, Hv, kSegSinImg);
+            float* sin = A.sin + (long long)(s - 1) * A.ss + unit;
+            uint8_t* img = A.img + ((long long)(s - 1) * A.ss + unit) * 4;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int r = row0 + ty * 4 + i;
@@ -87,7 +109,7 @@ gdn_prefill_combine_kernel(float* final_state, uint8_t* __restrict__ ws, WsLayou
                     make_uint2(pack_bf16x2(acc[i][0], acc[i][1]), pack_bf16x2(acc[i][2], acc[i][3]));
             }
         }
-        const float* H = reinterpret_cast<const float*>(ws + seg_block_offset(L, n, s, h, Hv, kSegH));
+        const float* H = A.H + (long long)(s - 1) * A.ss + unit;
         float4 hrow[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) hrow[i] = *reinterpret_cast<const float4*>(H + (size_t)(row0 + ty * 4 + i) * kD + tx * 4);
@@ -123,11 +145,11 @@ gdn_prefill_combine_kernel(float* final_state, uint8_t* __restrict__ ws, WsLayou
         }
     }
     if (*abort_flag) {
-        if (tid == 0) atomicExch(reinterpret_cast<int*>(ws), kStatusTimeout);
+        if (tid == 0 && A.status) atomicExch(A.status, kStatusTimeout);
         return;
     }
-    if (final_state) {
-        float* fin = final_state + ((size_t)n * Hv + h) * kD * kD;
+    if (A.fin) {
+        float* fin = A.fin + ((size_t)n * Hv + h) * kD * kD;
 #pragma unroll
         for (int i = 0; i < 4; ++i)
             *reinterpret_cast<float4*>(fin + (size_t)(row0 + ty * 4 + i) * kD + tx * 4) =
@@ -147,19 +169,32 @@ constexpr uint32_t FX_BAR = 98304;          // mbarriers, TMEM slot, abort flag
 constexpr uint32_t kFixSmem = FX_BAR + 64 + 1024;
 constexpr int kFixTokens = 128;
 
+// `cu` set: one run per sequence, tokens [cu[n], cu[n+1]), S_in image of (n, h) at img + (n Hv + h) 32 KB.
+// `cu` NULL: runs 1 .. segs-1 of every sequence from the chunk table in the workspace.
 __global__ void __launch_bounds__(128)
 gdn_prefill_fixup_kernel(const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_qt,
-                         uint16_t* __restrict__ out, uint8_t* __restrict__ ws, WsLayout L, int Hv, int segs) {
-    const int n = blockIdx.z / (segs - 1), s = blockIdx.z % (segs - 1) + 1, h = blockIdx.y;
-    const int tid = threadIdx.x, warp = tid >> 5;
-    const int* chunk_off = reinterpret_cast<const int*>(ws + L.off_chunk_off);
-    const int4* chunk_info = reinterpret_cast<const int4*>(ws + L.off_chunk_info);
-    int first, count;
-    segment_range(chunk_off[n + 1] - chunk_off[n], segs, s, first, count);
-    if (count <= 0) return;
-    const int c0 = chunk_off[n] + first;
-    const int t_begin = chunk_info[c0].y;
-    const int t_end = chunk_info[c0 + count - 1].y + chunk_info[c0 + count - 1].z;
+                         uint16_t* __restrict__ out, uint8_t* __restrict__ ws, WsLayout L, int Hv, int segs,
+                         const int* __restrict__ cu, const uint8_t* __restrict__ img_base) {
+    const int tid = threadIdx.x, warp = tid >> 5, h = blockIdx.y;
+    int t_begin, t_end;
+    const uint8_t* img;
+    if (cu) {
+        const int n = blockIdx.z;
+        t_begin = cu[n];
+        t_end = cu[n + 1];
+        img = img_base + ((size_t)n * Hv + h) * 32768;
+    } else {
+        const int n = blockIdx.z / (segs - 1), s = blockIdx.z % (segs - 1) + 1;
+        const int* chunk_off = reinterpret_cast<const int*>(ws + L.off_chunk_off);
+        const int4* chunk_info = reinterpret_cast<const int4*>(ws + L.off_chunk_info);
+        int first, count;
+        segment_range(chunk_off[n + 1] - chunk_off[n], segs, s, first, count);
+        if (count <= 0) return;
+        const int c0 = chunk_off[n] + first;
+        t_begin = chunk_info[c0].y;
+        t_end = chunk_info[c0 + count - 1].y + chunk_info[c0 + count - 1].z;
+        img = ws + seg_block_offset(L, n, s, h, Hv, kSegSinImg);
+    }
     const int t0 = t_begin + blockIdx.x * kFixTokens;
     if (t0 >= t_end) return;
     const int rows = min(kFixTokens, t_end - t0);
@@ -176,7 +211,7 @@ gdn_prefill_fixup_kernel(const __grid_constant__ CUtensorMap map_out, const __gr
         *abort_flag = 0;
         mbar_fence_init();
         mbar_expect_tx(bar_load, 3u * 32768u);
-        bulk_load(smem + FX_B, ws + seg_block_offset(L, n, s, h, Hv, kSegSinImg), 32768, bar_load);
+        bulk_load(smem + FX_B, img, 32768, bar_load);
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb)
 #pragma unroll
@@ -251,10 +286,7 @@ gdn_prefill_fixup_kernel(const __grid_constant__ CUtensorMap map_out, const __gr
     }
 }
 
-cudaError_t launch_prefill_scan(const CUtensorMap& mout, const CUtensorMap& mqt, void* out, float* final_state,
-                                uint8_t* ws, const WsLayout& L, int num_seqs, int max_seqlen, int Hv, int segs,
-                                cudaStream_t st) {
-    if (segs <= 1) return cudaSuccess;
+static cudaError_t scan_attrs() {
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(gdn_prefill_fixup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFixSmem);
@@ -263,20 +295,102 @@ cudaError_t launch_prefill_scan(const CUtensorMap& mout, const CUtensorMap& mqt,
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
+    return cudaSuccess;
+}
+
+cudaError_t launch_prefill_scan(const CUtensorMap& mout, const CUtensorMap& mqt, void* out, float* final_state,
+                                uint8_t* ws, const WsLayout& L, int num_seqs, int max_seqlen, int Hv, int segs,
+                                cudaStream_t st) {
+    if (segs <= 1) return cudaSuccess;
+    if (cudaError_t e = scan_attrs()) return e;
     const dim3 cgrid((unsigned)(num_seqs * Hv), kD / kCombineRows);
     // two P buffers need a whole SM per CTA: worth it when there are several steps and the grid is small
     const int nbuf = (segs > 2 && (long long)cgrid.x * cgrid.y <= kAssumedSMs) ? 2 : 1;
+    ScanArgs A;
+    const long long blk = (long long)(kSegBlockBytes / sizeof(float));
+    float* seg0 = reinterpret_cast<float*>(ws + L.off_seg);
+    A.ss = (long long)Hv * kSegBlocks * blk;
+    A.sn = (long long)(L.seg_cap - 1) * Hv * kSegBlocks * blk;
+    A.sh = (long long)kSegBlocks * blk;
+    A.x0 = seg0 + kSegSin * blk;  // run 1's entering state = run 0's final state
+    A.x_sn = A.sn;
+    A.x_sh = A.sh;
+    A.P = seg0 + kSegP * blk;
+    A.H = seg0 + kSegH * blk;
+    A.sin = seg0 + kSegSin * blk;
+    A.img = ws + L.off_seg + kSegSinImg * kSegBlockBytes;
+    A.fin = final_state;
+    A.steps = segs - 1;
+    A.chunk_off = reinterpret_cast<const int*>(ws + L.off_chunk_off);
+    A.segs = segs;
+    A.status = reinterpret_cast<int*>(ws);
     // states entering runs 2.. come out of the combine; with two runs the fix-up only needs run 0's
     // final state, so the combine (then only the final state) goes last
-    if (segs > 2)
-        gdn_prefill_combine_kernel<<<cgrid, 128, combine_smem(nbuf), st>>>(final_state, ws, L, Hv, segs, nbuf);
+    if (segs > 2) gdn_prefill_combine_kernel<<<cgrid, 128, combine_smem(nbuf), st>>>(A, Hv, nbuf);
     const int max_chunks = (max_seqlen + kChunk - 1) / kChunk;
     const int seg_chunks = (max_chunks + segs - 1) / segs;
     const dim3 fgrid((unsigned)((seg_chunks * kChunk + kFixTokens - 1) / kFixTokens), (unsigned)Hv,
                      (unsigned)(num_seqs * (segs - 1)));
-    gdn_prefill_fixup_kernel<<<fgrid, 128, kFixSmem, st>>>(mout, mqt, (uint16_t*)out, ws, L, Hv, segs);
-    if (segs == 2 && final_state)
-        gdn_prefill_combine_kernel<<<cgrid, 128, combine_smem(nbuf), st>>>(final_state, ws, L, Hv, segs, nbuf);
+    gdn_prefill_fixup_kernel<<<fgrid, 128, kFixSmem, st>>>(mout, mqt, (uint16_t*)out, ws, L, Hv, segs, nullptr, nullptr);
+    if (segs == 2 && final_state) gdn_prefill_combine_kernel<<<cgrid, 128, combine_smem(nbuf), st>>>(A, Hv, nbuf);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same two kernels behind the sequence-parallel building blocks of the C ABI.
+
+// fp32 [N][Hv][128][128] -> bf16 operand tiles (two swizzled [128 v][64 k] tiles per (n, h))
+__global__ void __launch_bounds__(128) gdn_state_image_kernel(const float* __restrict__ S, uint8_t* __restrict__ img) {
+    const float* src = S + (size_t)blockIdx.x * kD * kD;
+    uint8_t* dst = img + (size_t)blockIdx.x * 32768;
+#pragma unroll 4
+    for (int it = 0; it < 16; ++it) {
+        const int piece = it * 128 + threadIdx.x, r = piece >> 4, c = piece & 15;
+        const float4 x = *reinterpret_cast<const float4*>(src + (size_t)r * kD + c * 8);
+        const float4 y = *reinterpret_cast<const float4*>(src + (size_t)r * kD + c * 8 + 4);
+        *reinterpret_cast<uint4*>(dst + (c >> 3) * 16384 + swz((uint32_t)r, (uint32_t)(c & 7))) =
+            make_uint4(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w), pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
+    }
+}
+
+// S_out[n][h] = (...((S0 P_0 + H_0) P_1 + H_1)...) over `steps` blocks laid out [steps][N][Hv][128][128]
+cudaError_t launch_state_scan(const float* S0, const float* P, const float* H, int steps, float* S_out, int num_seqs,
+                              int Hv, cudaStream_t st) {
+    if (cudaError_t e = scan_attrs()) return e;
+    const dim3 cgrid((unsigned)(num_seqs * Hv), kD / kCombineRows);
+    const int nbuf = (steps > 1 && (long long)cgrid.x * cgrid.y <= kAssumedSMs) ? 2 : 1;
+    ScanArgs A;
+    const long long blk = (long long)kD * kD;
+    A.x0 = S0;
+    A.x_sn = (long long)Hv * blk;
+    A.x_sh = blk;
+    A.P = P;
+    A.H = H;
+    A.ss = (long long)num_seqs * Hv * blk;
+    A.sn = (long long)Hv * blk;
+    A.sh = blk;
+    A.sin = nullptr;
+    A.img = nullptr;
+    A.fin = S_out;
+    A.steps = steps;
+    A.chunk_off = nullptr;
+    A.segs = 0;
+    A.status = nullptr;
+    gdn_prefill_combine_kernel<<<cgrid, 128, combine_smem(nbuf), st>>>(A, Hv, nbuf);
+    return cudaGetLastError();
+}
+
+// out[t][h][:] += S_in[n][h] qt[t][h][:] for every token of every sequence
+cudaError_t launch_prefill_apply(const CUtensorMap& mout, const CUtensorMap& mqt, const float* S_in, void* out,
+                                 const int32_t* cu_seqlens, int num_seqs, int max_seqlen, int Hv, uint8_t* ws,
+                                 cudaStream_t st) {
+    if (cudaError_t e = scan_attrs()) return e;
+    cudaMemsetAsync(ws, 0, 8, st);  // device status word
+    uint8_t* img = ws + 1024;
+    gdn_state_image_kernel<<<(unsigned)(num_seqs * Hv), 128, 0, st>>>(S_in, img);
+    const dim3 fgrid((unsigned)((max_seqlen + kFixTokens - 1) / kFixTokens), (unsigned)Hv, (unsigned)num_seqs);
+    WsLayout L = {};
+    gdn_prefill_fixup_kernel<<<fgrid, 128, kFixSmem, st>>>(mout, mqt, (uint16_t*)out, ws, L, Hv, 2, cu_seqlens, img);
     return cudaGetLastError();
 }
 

@@ -87,13 +87,27 @@ cudaError_t launch_prefill_prep(const int32_t* cu_seqlens, int num_seqs, int tot
 cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, const float* g, const float* beta,
                                  const float* A_log, const float* dt_bias, uint8_t* ws, const WsLayout& L, int Hqk,
                                  int Hv, cudaStream_t st);
+// Destinations of the chain kernel's partial mode (gdn_prefill_partial): all NULL = normal mode.
+struct ChainPartial {
+    float* H;      // fp32 [N][Hv][128][128]: state reached from the zero state
+    float* P;      // fp32 [N][Hv][128][128]: transition (state reached from the identity with v = 0)
+    uint16_t* qt;  // bf16 [T][Hv][128]: M_t q_t
+};
+
 // `segs` > 1 splits every sequence into that many runs of chunks (see gdn_prefill_scan.cu).
 cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                                  const float* initial_state, void* out, float* final_state, uint8_t* ws,
-                                 const WsLayout& L, int num_seqs, int Hqk, int Hv, int segs, cudaStream_t st);
+                                 const WsLayout& L, int num_seqs, int Hqk, int Hv, int segs, const ChainPartial& part,
+                                 cudaStream_t st);
 cudaError_t launch_prefill_scan(const CUtensorMap& mout, const CUtensorMap& mqt, void* out, float* final_state,
                                 uint8_t* ws, const WsLayout& L, int num_seqs, int max_seqlen, int Hv, int segs,
                                 cudaStream_t st);
+
+cudaError_t launch_state_scan(const float* S0, const float* P, const float* H, int steps, float* S_out, int num_seqs,
+                              int Hv, cudaStream_t st);
+cudaError_t launch_prefill_apply(const CUtensorMap& mout, const CUtensorMap& mqt, const float* S_in, void* out,
+                                 const int32_t* cu_seqlens, int num_seqs, int max_seqlen, int Hv, uint8_t* ws,
+                                 cudaStream_t st);
 
 // Chunks [first, first + count) of segment `s` when a sequence of `nchunks` chunks is cut into `segs`.
 __host__ __device__ inline void segment_range(int nchunks, int segs, int s, int& first, int& count) {
