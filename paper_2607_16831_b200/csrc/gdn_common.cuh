@@ -1,5 +1,6 @@
 // Shared device/host helpers of libgdn (internal; the public boundary is include/gdn.h).
 #pragma once
+#include <cstdlib>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -51,5 +52,40 @@ __device__ __forceinline__ void raw_gates(float a, float b, float A_log, float d
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Programmatic dependent launch.  A kernel launched with launch_pdl may be scheduled while the
+// kernel before it in the stream is still running (once every CTA of that kernel has called
+// pdl_launch_dependents or exited); it must call pdl_wait before it reads or writes anything the
+// earlier kernel touches.  pdl_wait returns when the earlier grid has completed and its writes are
+// visible, so stream order is kept; what is saved is the drain-and-refill gap between two kernels.
+// Both calls are no-ops for a kernel that was launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// GDN_NO_PDL=1 in the environment launches everything the ordinary way.
+inline bool pdl_enabled() {
+    static int state = -1;
+    if (state < 0) {
+        const char* e = getenv("GDN_NO_PDL");
+        state = (e && e[0] == '1') ? 0 : 1;
+    }
+    return state == 1;
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 }  // namespace gdn

@@ -75,6 +75,9 @@ gdn_decode_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k
                   const float* __restrict__ beta, const float* __restrict__ A_log,
                   const float* __restrict__ dt_bias, const float* s_in, float* s_out,
                   uint16_t* __restrict__ out, int Hqk, int Hv, int split) {
+    // the kernel before this one in the stream may have produced the tokens or the state
+    pdl_wait();
+    pdl_launch_dependents();
     const int cta = blockIdx.x;
     const int part = cta % split;
     const int bh = cta / split;  // b*Hv + h
@@ -120,10 +123,9 @@ static cudaError_t launch(const void* q, const void* k, const void* v, const flo
     constexpr int split = kD / (WARPS * 4 * NB);
     static_assert(split >= 1 && split * WARPS * 4 * NB == kD, "rows must tile the head");
     const long long ctas = (long long)B * Hv * split;
-    gdn_decode_kernel<NB, WARPS><<<(unsigned)ctas, WARPS * 32, 0, st>>>(
-        (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta, A_log, dt_bias, s_in, s_out, (uint16_t*)out,
-        Hqk, Hv, split);
-    return cudaGetLastError();
+    return launch_pdl(gdn_decode_kernel<NB, WARPS>, dim3((unsigned)ctas), dim3(WARPS * 32), 0, st,
+                      (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta, A_log, dt_bias, s_in, s_out,
+                      (uint16_t*)out, Hqk, Hv, split);
 }
 
 // Launch-shape table.  `variant` < 0 picks from the batch size: below ~16 items the
@@ -163,6 +165,8 @@ gdn_decode_multi_kernel(const uint16_t* __restrict__ q, const uint16_t* __restri
                         const uint16_t* __restrict__ v, const float* __restrict__ g,
                         const float* __restrict__ beta, const float* s_in, float* s_out,
                         uint16_t* __restrict__ out, int T, int Hqk, int Hv, int split) {
+    pdl_wait();
+    pdl_launch_dependents();
     const int cta = blockIdx.x;
     const int part = cta % split;
     const int bh = cta / split;
@@ -246,14 +250,14 @@ cudaError_t decode_multi_dispatch(const void* q, const void* k, const void* v, c
                                   cudaStream_t st) {
     if (B <= 2) {
         constexpr int NB = 1, WARPS = 1, split = kD / (WARPS * 4 * NB);
-        gdn_decode_multi_kernel<NB, WARPS><<<(unsigned)((long long)B * Hv * split), WARPS * 32, 0, st>>>(
-            (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta, s_in, s_out, (uint16_t*)out, T, Hqk,
-            Hv, split);
+        return launch_pdl(gdn_decode_multi_kernel<NB, WARPS>, dim3((unsigned)((long long)B * Hv * split)),
+                          dim3(WARPS * 32), 0, st, (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta,
+                          s_in, s_out, (uint16_t*)out, T, Hqk, Hv, split);
     } else {
         constexpr int NB = 2, WARPS = 4, split = kD / (WARPS * 4 * NB);
-        gdn_decode_multi_kernel<NB, WARPS><<<(unsigned)((long long)B * Hv * split), WARPS * 32, 0, st>>>(
-            (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta, s_in, s_out, (uint16_t*)out, T, Hqk,
-            Hv, split);
+        return launch_pdl(gdn_decode_multi_kernel<NB, WARPS>, dim3((unsigned)((long long)B * Hv * split)),
+                          dim3(WARPS * 32), 0, st, (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta,
+                          s_in, s_out, (uint16_t*)out, T, Hqk, Hv, split);
     }
     return cudaGetLastError();
 }
