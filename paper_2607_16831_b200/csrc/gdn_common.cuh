@@ -62,6 +62,16 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Function attributes (dynamic shared memory above 48 KB) are per device: returns true the first
+// time it is asked about `flags` on the current device, so the caller sets them then.
+inline bool first_use_on_device(bool (&flags)[64]) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;  // unknown: set them again
+    if (flags[dev]) return false;
+    flags[dev] = true;
+    return true;
+}
+
 // GDN_NO_PDL=1 in the environment launches everything the ordinary way.
 inline bool pdl_enabled() {
     static int state = -1;

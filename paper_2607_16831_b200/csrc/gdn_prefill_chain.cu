@@ -545,12 +545,11 @@ cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, c
                                  const float* initial_state, void* out, float* final_state, uint8_t* ws,
                                  const WsLayout& L, int num_seqs, int Hqk, int Hv, int segs, const ChainPartial& part,
                                  cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
+    static bool attr_done[64];
+    if (first_use_on_device(attr_done)) {
         cudaError_t e = cudaFuncSetAttribute(gdn_prefill_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kChainSmem);
         if (e != cudaSuccess) return e;
-        attr_done = true;
     }
     const int per_seq = part.H ? 2 : 2 * segs - 1;
     gdn_prefill_chain_kernel<<<(unsigned)((long long)num_seqs * per_seq * Hv), kChainThreads, kChainSmem, st>>>(

@@ -439,12 +439,11 @@ cudaError_t launch_prefill_prep(const int32_t* cu_seqlens, int num_seqs, int tot
 cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, const float* g, const float* beta,
                                  const float* A_log, const float* dt_bias, uint8_t* ws, const WsLayout& L, int Hqk,
                                  int Hv, cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
+    static bool attr_done[64];
+    if (first_use_on_device(attr_done)) {
         cudaError_t e = cudaFuncSetAttribute(gdn_prefill_intra_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kIntraSmem);
         if (e != cudaSuccess) return e;
-        attr_done = true;
     }
     const int G = Hv / Hqk;
     dim3 grid(L.nc_max, Hqk * ((G + 1) / 2));

@@ -63,6 +63,25 @@ def test_host_side_argument_checks(gdn):
     a = list(args); a[0] = odd
     assert L.gdn_prefill(*a, 100, 2, 60, 16, 32, 128, 128, fake, 1 << 30, None) == 5
     assert L.gdn_prefill_recurrent(*args, 100, 2, 101, 16, 32, 128, 128, None) == 2
+    # sequence-parallel building blocks
+    pa = [fake] * 10
+    assert L.gdn_prefill_partial(*pa, 0, 0, 0, 16, 32, 128, 128, None, 0, None) == 0
+    assert L.gdn_prefill_partial(*pa, 100, 2, 101, 16, 32, 128, 128, fake, 1 << 30, None) == 2
+    assert L.gdn_prefill_partial(*pa, 100, 2, 60, 16, 32, 64, 128, fake, 1 << 30, None) == 3
+    a = list(pa); a[5] = None
+    assert L.gdn_prefill_partial(*a, 100, 2, 60, 16, 32, 128, 128, fake, 1 << 30, None) == 1   # cu_seqlens NULL
+    a = list(pa); a[2] = odd
+    assert L.gdn_prefill_partial(*a, 100, 2, 60, 16, 32, 128, 128, fake, 1 << 30, None) == 5
+    assert L.gdn_state_scan(fake, fake, fake, 3, fake, 0, 32, 128, 128, None) == 0             # no sequences
+    assert L.gdn_state_scan(fake, fake, fake, -1, fake, 1, 32, 128, 128, None) == 2
+    assert L.gdn_state_scan(fake, fake, fake, 3, None, 1, 32, 128, 128, None) == 1
+    assert L.gdn_state_scan(fake, None, fake, 3, fake, 1, 32, 128, 128, None) == 1
+    assert L.gdn_state_scan(fake, odd, fake, 3, fake, 1, 32, 128, 128, None) == 5
+    assert L.gdn_state_scan(fake, fake, fake, 3, fake, 1, 32, 128, 64, None) == 3
+    assert L.gdn_prefill_apply(fake, fake, fake, fake, 0, 0, 0, 32, 128, 128, None, 0, None) == 0
+    assert L.gdn_prefill_apply(fake, fake, fake, fake, 100, 2, 101, 32, 128, 128, fake, 1 << 30, None) == 2
+    assert L.gdn_prefill_apply(None, fake, fake, fake, 100, 2, 60, 32, 128, 128, fake, 1 << 30, None) == 1
+    assert L.gdn_prefill_apply(fake, fake, odd, fake, 100, 2, 60, 32, 128, 128, fake, 1 << 30, None) == 5
 
 
 def test_workspace_size_grows_with_tokens(gdn):
