@@ -15,7 +15,7 @@ cudaError_t decode_multi_dispatch(const void* q, const void* k, const void* v, c
 cudaError_t prefill_recurrent_dispatch(const void* q, const void* k, const void* v, const float* g,
                                        const float* beta, const int32_t* cu_seqlens, const float* initial_state,
                                        void* out, float* final_state, int total_tokens, int num_seqs, int Hqk,
-                                       int Hv, cudaStream_t st);
+                                       int Hv, int* status_word, cudaStream_t st);
 size_t prefill_chunked_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv, bool allow_split);
 cudaError_t prefill_partial_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
                                      const int32_t* cu_seqlens, void* out0, void* qt, float* H, float* P,
@@ -108,18 +108,19 @@ static int check_prefill(const void* q, const void* k, const void* v, const floa
 
 // Short-sequence dispatch of gdn_prefill.  When no sequence is longer than one chunk the chunked
 // path pays for whole 64-token chunks and three dependent launches (about 27 us even for a few
-// tokens), while the token-serial kernel costs about 0.6 us per token of the longest sequence,
-// times the number of waves its (sequence, head) units need.  Both models are fits to
-// measurements on B200 over 1..64 sequences of 4..128 tokens at 8 and 32 value heads; the faster
-// one by the model is used.  GDN_PREFILL_SHORT_FALLBACK=0 (environment) keeps the chunked path.
+// tokens, 13 us + 0.09 us per (sequence, head) chain beyond that), while the token-serial kernel
+// costs about 0.45 us per token of the longest sequence, or 0.006 us per token and chain once the
+// chains fill the GPU.  Both models are fits to measurements on B200 over 1..64 sequences of 4..128
+// tokens at 8 and 32 value heads; the faster one by the model is used.
+// GDN_PREFILL_SHORT_FALLBACK=0 (environment) keeps the chunked path.
 static bool prefer_token_serial(int num_seqs, int Hv, int max_seqlen) {
     if (max_seqlen > kChunk) return false;
     if (const char* env = getenv("GDN_PREFILL_SHORT_FALLBACK"))
         if (env[0] == '0') return false;
     const double chains = (double)num_seqs * Hv;
-    const double waves = chains > 96.0 ? chains / 96.0 : 1.0;
-    const double t_serial = 2.0 + 0.014 * chains + 0.6 * max_seqlen * waves;
-    const double t_chunked = 0.098 * chains > 27.0 ? 0.098 * chains : 27.0;
+    const double per_token = 0.006 * chains > 0.45 ? 0.006 * chains : 0.45;
+    const double t_serial = 1.3 + 0.012 * chains + per_token * max_seqlen;
+    const double t_chunked = 13.0 + 0.092 * chains > 27.0 ? 13.0 + 0.092 * chains : 27.0;
     return t_serial < t_chunked;
 }
 
@@ -195,10 +196,9 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
         return GDN_ERR_WORKSPACE;
     if (prefer_token_serial(num_seqs, Hv, max_seqlen)) {
-        // the device status word the chunked kernels would have cleared
-        cudaMemsetAsync(workspace, 0, 8, (cudaStream_t)stream);
         return cuda_status(prefill_recurrent_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
-                                                      total_tokens, num_seqs, Hqk, Hv, (cudaStream_t)stream),
+                                                      total_tokens, num_seqs, Hqk, Hv, static_cast<int*>(workspace),
+                                                      (cudaStream_t)stream),
                            "gdn_prefill (token-serial)");
     }
     return cuda_status(prefill_chunked_dispatch(q, k, v, g, beta, nullptr, nullptr, cu_seqlens, initial_state, out,
@@ -242,7 +242,7 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const flo
         return rc;
     if (nothing) return GDN_OK;
     return cuda_status(prefill_recurrent_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
-                                                  total_tokens, num_seqs, Hqk, Hv, (cudaStream_t)stream),
+                                                  total_tokens, num_seqs, Hqk, Hv, nullptr, (cudaStream_t)stream),
                        "gdn_prefill_recurrent");
 }
 

@@ -21,7 +21,9 @@ gdn_prefill_recurrent_kernel(const uint16_t* __restrict__ q, const uint16_t* __r
                              const uint16_t* __restrict__ v, const float* __restrict__ g,
                              const float* __restrict__ beta, const int32_t* __restrict__ cu_seqlens,
                              const float* initial_state, uint16_t* __restrict__ out, float* final_state,
-                             int total_tokens, int Hqk, int Hv, int split) {
+                             int total_tokens, int Hqk, int Hv, int split, int* status_word) {
+    // standing in for the chunked kernels: clear the workspace's device status word as they would
+    if (status_word && blockIdx.x == 0 && threadIdx.x == 0) *status_word = 0;
     const int part = blockIdx.x % split;
     const int h = (blockIdx.x / split) % Hv;
     const int n = blockIdx.x / split / Hv;
@@ -124,17 +126,33 @@ gdn_prefill_recurrent_kernel(const uint16_t* __restrict__ q, const uint16_t* __r
     }
 }
 
-cudaError_t prefill_recurrent_dispatch(const void* q, const void* k, const void* v, const float* g,
-                                       const float* beta, const int32_t* cu_seqlens, const float* initial_state,
-                                       void* out, float* final_state, int total_tokens, int num_seqs, int Hqk,
-                                       int Hv, cudaStream_t st) {
-    constexpr int NB = 2, WARPS = 2;
+template <int NB, int WARPS>
+static cudaError_t launch_recurrent(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                                    const int32_t* cu_seqlens, const float* initial_state, void* out,
+                                    float* final_state, int total_tokens, int num_seqs, int Hqk, int Hv,
+                                    int* status_word, cudaStream_t st) {
     constexpr int split = kD / (WARPS * 4 * NB);
     const unsigned grid = (unsigned)((long long)split * Hv * num_seqs);
     gdn_prefill_recurrent_kernel<NB, WARPS><<<grid, WARPS * 32, 0, st>>>(
         (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta, cu_seqlens, initial_state,
-        (uint16_t*)out, final_state, total_tokens, Hqk, Hv, split);
+        (uint16_t*)out, final_state, total_tokens, Hqk, Hv, split, status_word);
     return cudaGetLastError();
+}
+
+cudaError_t prefill_recurrent_dispatch(const void* q, const void* k, const void* v, const float* g,
+                                       const float* beta, const int32_t* cu_seqlens, const float* initial_state,
+                                       void* out, float* final_state, int total_tokens, int num_seqs, int Hqk,
+                                       int Hv, int* status_word, cudaStream_t st) {
+    // Launch shape by the number of (sequence, head) chains, from a sweep on B200 (1-64 sequences of
+    // 8 and 32 tokens, 8 and 32 value heads): few chains want many small warps' worth of rows each
+    // (the token loop is latency-bound: fewer rows per warp = a shorter loop body); thousands of
+    // chains want one-warp CTAs (more CTAs resident per SM); everything between, four warps of 8 rows.
+#define GDN_REC_ARGS q, k, v, g, beta, cu_seqlens, initial_state, out, final_state, total_tokens, num_seqs, Hqk, Hv, status_word, st
+    const long long chains = (long long)num_seqs * Hv;
+    if (chains <= 16) return launch_recurrent<1, 2>(GDN_REC_ARGS);
+    if (chains >= 1024) return launch_recurrent<2, 1>(GDN_REC_ARGS);
+    return launch_recurrent<2, 4>(GDN_REC_ARGS);
+#undef GDN_REC_ARGS
 }
 
 }  // namespace gdn
