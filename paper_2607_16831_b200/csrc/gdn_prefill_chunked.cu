@@ -69,14 +69,17 @@ cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v
                                      bool allow_split, cudaStream_t st) {
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     const WsLayout L = ws_layout(total_tokens, num_seqs, Hv, allow_split);
-    cudaError_t e = launch_prefill_prep(cu_seqlens, num_seqs, total_tokens, ws, L, st);
+    // with few sequences the intra-chunk kernel builds the chunk table itself (one launch less)
+    const bool no_prep = total_tokens > 0 && num_seqs <= kMaxSeqsWithoutPrep;
+    cudaError_t e = no_prep ? cudaSuccess : launch_prefill_prep(cu_seqlens, num_seqs, total_tokens, ws, L, st);
     if (e != cudaSuccess) return e;
     if (total_tokens > 0) {
         CUtensorMap mq, mk, mv;
         if (!make_map(&mq, q, total_tokens, Hqk) || !make_map(&mk, k, total_tokens, Hqk) ||
             !make_map(&mv, v, total_tokens, Hv))
             return cudaErrorUnknown;
-        e = launch_prefill_intra(mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv, st);
+        e = launch_prefill_intra(mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv, no_prep ? cu_seqlens : nullptr, num_seqs,
+                                 total_tokens, st);
         if (e != cudaSuccess) return e;
         const int segs = choose_segments(L, num_seqs, Hv, max_seqlen);
         e = launch_prefill_chain(mq, mk, mv, initial_state, out, final_state, ws, L, num_seqs, Hqk, Hv, segs,
@@ -116,7 +119,7 @@ cudaError_t prefill_partial_dispatch(const void* q, const void* k, const void* v
         if (!make_map(&mq, q, total_tokens, Hqk) || !make_map(&mk, k, total_tokens, Hqk) ||
             !make_map(&mv, v, total_tokens, Hv))
             return cudaErrorUnknown;
-        e = launch_prefill_intra(mq, mk, g, beta, nullptr, nullptr, ws, L, Hqk, Hv, st);
+        e = launch_prefill_intra(mq, mk, g, beta, nullptr, nullptr, ws, L, Hqk, Hv, nullptr, num_seqs, total_tokens, st);
         if (e != cudaSuccess) return e;
     } else {
         // no tensor to describe; every sequence is empty and the chain CTAs return before using the maps

@@ -103,16 +103,65 @@ __global__ void __launch_bounds__(kIntraThreads, 4)
 gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const float* __restrict__ g, const float* __restrict__ beta,
                          const float* __restrict__ A_log, const float* __restrict__ dt_bias,
-                         uint8_t* __restrict__ ws, WsLayout L, int Hqk, int Hv) {
+                         uint8_t* __restrict__ ws, WsLayout L, int Hqk, int Hv, const int32_t* __restrict__ cu,
+                         int num_seqs, int total_tokens) {
     const int c = blockIdx.x;
-    const int* hdr = reinterpret_cast<const int*>(ws);
-    if (c >= hdr[1]) return;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    int t0, len;
+    if (cu) {
+        // Few sequences: no chunk-table kernel ran.  Every CTA finds its chunk by walking cu_seqlens
+        // (one round trip: the loads are independent), and the first CTA leaves the tables the later
+        // kernels read -- what gdn_prefill_prep_kernel would have written.
+        int run = 0;
+        t0 = 0;
+        len = -1;
+        for (int n = 0; n < num_seqs; ++n) {
+            const int a = max(0, min(cu[n], total_tokens)), b = max(a, min(cu[n + 1], total_tokens));
+            const int nch = (b - a + kChunk - 1) / kChunk;
+            if (c >= run && c < run + nch) {
+                t0 = a + (c - run) * kChunk;
+                len = min(kChunk, b - t0);
+            }
+            run += nch;
+        }
+        if (blockIdx.x == 0 && blockIdx.y == 0) {
+            int* hdr_w = reinterpret_cast<int*>(ws);
+            int* chunk_off = reinterpret_cast<int*>(ws + L.off_chunk_off);
+            int* seq_order = reinterpret_cast<int*>(ws + L.off_seq_order);
+            int4* chunk_info = reinterpret_cast<int4*>(ws + L.off_chunk_info);
+            const int total = min(run, L.nc_max);
+            if (tid == 0) {
+                hdr_w[0] = 0;
+                hdr_w[1] = total;
+                chunk_off[num_seqs] = total;
+            }
+            for (int n = tid; n < num_seqs; n += kIntraThreads) {
+                int base = 0, rank = 0;
+                const int a = max(0, min(cu[n], total_tokens)), b = max(a, min(cu[n + 1], total_tokens));
+                for (int m = 0; m < num_seqs; ++m) {
+                    const int am = max(0, min(cu[m], total_tokens)), bm = max(am, min(cu[m + 1], total_tokens));
+                    if (m < n) base += (bm - am + kChunk - 1) / kChunk;
+                    rank += (bm - am > b - a) || (bm - am == b - a && m < n);
+                }
+                chunk_off[n] = min(base, L.nc_max);
+                seq_order[rank] = n;  // longest first
+                const int nch = (b - a + kChunk - 1) / kChunk;
+                for (int j = 0; j < nch; ++j)
+                    if (base + j < L.nc_max)
+                        chunk_info[base + j] = make_int4(n, a + j * kChunk, min(kChunk, b - a - j * kChunk), j);
+            }
+        }
+        if (len < 0 || c >= L.nc_max) return;
+    } else {
+        const int* hdr = reinterpret_cast<const int*>(ws);
+        if (c >= hdr[1]) return;
+        const int4 info = reinterpret_cast<const int4*>(ws + L.off_chunk_info)[c];
+        t0 = info.y;
+        len = info.z;
+    }
     const int G = Hv / Hqk;
     const int npairs = (G + 1) / 2;
     const int hq = blockIdx.y / npairs, p = blockIdx.y % npairs;
-    const int4 info = reinterpret_cast<const int4*>(ws + L.off_chunk_info)[c];
-    const int t0 = info.y, len = info.z;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int hh = tid >> 6, i = tid & 63;  // role in the gate / solve / W phases: head of the pair, row
     const int nh = min(2, G - 2 * p);
     const int h = hq * G + 2 * p + hh;      // this thread's value head in those phases
@@ -438,7 +487,8 @@ cudaError_t launch_prefill_prep(const int32_t* cu_seqlens, int num_seqs, int tot
 
 cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, const float* g, const float* beta,
                                  const float* A_log, const float* dt_bias, uint8_t* ws, const WsLayout& L, int Hqk,
-                                 int Hv, cudaStream_t st) {
+                                 int Hv, const int32_t* cu_if_no_table, int num_seqs, int total_tokens,
+                                 cudaStream_t st) {
     static bool attr_done[64];
     if (first_use_on_device(attr_done)) {
         cudaError_t e = cudaFuncSetAttribute(gdn_prefill_intra_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -447,7 +497,8 @@ cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, c
     }
     const int G = Hv / Hqk;
     dim3 grid(L.nc_max, Hqk * ((G + 1) / 2));
-    gdn_prefill_intra_kernel<<<grid, kIntraThreads, kIntraSmem, st>>>(mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv);
+    gdn_prefill_intra_kernel<<<grid, kIntraThreads, kIntraSmem, st>>>(mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv,
+                                                                      cu_if_no_table, num_seqs, total_tokens);
     return cudaGetLastError();
 }
 

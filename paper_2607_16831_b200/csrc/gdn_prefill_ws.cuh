@@ -84,9 +84,13 @@ __host__ __device__ __forceinline__ uint32_t swz(uint32_t r, uint32_t c16) {
 // Kernel launchers (defined next to their kernels).
 cudaError_t launch_prefill_prep(const int32_t* cu_seqlens, int num_seqs, int total_tokens, uint8_t* ws,
                                 const WsLayout& L, cudaStream_t st);
+// `cu_if_no_table` set: launch_prefill_prep did not run; the intra-chunk kernel derives the chunk table
+// from cu_seqlens itself and writes it for the later kernels (few sequences only: every CTA walks them).
+constexpr int kMaxSeqsWithoutPrep = 8;
 cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, const float* g, const float* beta,
                                  const float* A_log, const float* dt_bias, uint8_t* ws, const WsLayout& L, int Hqk,
-                                 int Hv, cudaStream_t st);
+                                 int Hv, const int32_t* cu_if_no_table, int num_seqs, int total_tokens,
+                                 cudaStream_t st);
 // Destinations of the chain kernel's partial mode (gdn_prefill_partial): all NULL = normal mode.
 struct ChainPartial {
     float* H;      // fp32 [N][Hv][128][128]: state reached from the zero state
