@@ -162,6 +162,13 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int G = Hv / Hqk;
     const int npairs = (G + 1) / 2;
     const int hq = blockIdx.y / npairs, p = blockIdx.y % npairs;
+#ifdef GDN_INTRA_PROFILE
+    // SM-clock stamps of thread 0 into the unused tail of this CTA's first scalar block (4-byte slots from byte 576)
+#define GDN_ISTAMP(slot) do { if (threadIdx.x == 0) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)c * Hv + hq * G + 2 * p) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
+#else
+#define GDN_ISTAMP(slot) do { } while (0)
+#endif
+    GDN_ISTAMP(0);
     const int hh = tid >> 6, i = tid & 63;  // role in the gate / solve / W phases: head of the pair, row
     const int nh = min(2, G - 2 * p);
     const int h = hq * G + 2 * p + hh;      // this thread's value head in those phases
@@ -258,6 +265,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         }
     }
     ok = __syncthreads_and(ok);
+    GDN_ISTAMP(1);
     if (ok) {
         tc_fence_after_sync();
         // per-token scalars of this thread's (head, row)
@@ -348,6 +356,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         tc_fence_before_sync();
         __syncthreads();  // B tiles and diagonal blocks complete; the accumulator of MMA1 is dead from here on
         tc_fence_after_sync();
+        GDN_ISTAMP(2);
 
         // ---- the blocked solve: z[jb][.] = columns 16 jb .. 16 jb + 15 of row i of T
         float z[4][16];
@@ -373,6 +382,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
                 for (int jj = 0; jj < mm; ++jj) rhs[jj] = fmaf(-dg[jj * 16 + mm], z[jb][mm], rhs[jj]);
             }
+            GDN_ISTAMP(3 + 2 * (3 - jb));
             if (jb > 0) {
                 // this block becomes a K step of the A operand (bf16 hi + lo) for the remaining steps
                 uint32_t zh[8], zl[8];
@@ -402,6 +412,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 ok = __syncthreads_and(ok);
                 if (!ok) break;
                 tc_fence_after_sync();
+                GDN_ISTAMP(4 + 2 * (3 - jb));
             }
         }
         if (ok) {
@@ -431,6 +442,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tc_fence_before_sync();
         }
         __syncthreads();
+        GDN_ISTAMP(11);
         // ---- MMA2: W (both heads) = [T''_a ; T''_b] K, K read MN-major from the TMA tiles
         if (ok && warp == 0) {
             tc_fence_after_sync();
@@ -443,6 +455,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             ok = mbar_wait_all(bar_mma2, 0, abort_flag);
         }
         ok = __syncthreads_and(ok);
+        GDN_ISTAMP(12);
     }
     if (ok) {
         tc_fence_after_sync();
@@ -467,6 +480,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         }
     }
 
+    GDN_ISTAMP(13);
     if (*abort_flag && tid == 0) atomicExch(reinterpret_cast<int*>(ws), kStatusTimeout);
     tc_fence_before_sync();
     __syncthreads();
