@@ -80,6 +80,9 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     // CTAs are handed out longest sequence first; within a sequence: run 0, then (zero, identity) per run.
     // Partial mode (part.H set, segs = 1): every sequence is one run that is walked from the zero state
     // and from the identity, results to the caller's H, P and qt.
+#ifdef GDN_CHAIN_PROFILE
+    const uint32_t t_entry = (uint32_t)clock64();
+#endif
     const bool partial = part.H != nullptr;
     const int per_seq = partial ? 2 : 2 * segs - 1;
     const int h = blockIdx.x % Hv, unit = blockIdx.x / Hv;
@@ -158,6 +161,11 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #define GDN_STAMP(c, slot) do { if (blockIdx.x == 0) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)(c) * Hv + h) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
 #else
 #define GDN_STAMP(c, slot) do { } while (0)
+#endif
+    if (tid == 0) GDN_STAMP(c_begin, 40);  // set-up done (tables read, barriers, tensor memory)
+#ifdef GDN_CHAIN_PROFILE
+    if (tid == 0 && blockIdx.x == 0)
+        reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)c_begin * Hv + h) * kScalBytes + 576)[43] = t_entry;
 #endif
 
     if (warp == 8) {
@@ -348,6 +356,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tc_fence_before_sync();
             warp_arrive(bars + B_SHI);
             warp_arrive(bars + B_STM);
+            if (tid == 0) GDN_STAMP(c_begin, 42);  // initial state in tensor memory
         }
         for (int ci = 0; ci < nchunks; ++ci) {
             const int c = c_begin + ci;
@@ -527,6 +536,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         }
     }
 
+    if (tid == 0) GDN_STAMP(c_begin, 41);  // this thread's role is finished
     // ---- unwind: on failure give copies in flight a moment to land, then release tensor memory
     if (*abort_flag) {
         const long long t_start = clock64();
