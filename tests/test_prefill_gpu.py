@@ -172,3 +172,13 @@ def test_prefill_malformed_cu_seqlens_stays_in_bounds():
     assert gdn.gdn_last_device_status(ws) == 0
     assert torch.all(out_buf[100:] == 7.0)
     assert torch.isfinite(fin).all()
+
+
+@pytest.mark.parametrize("gate_mean", [-4.0, -12.0])
+def test_prefill_strong_decay_underflows_cleanly(gate_mean):
+    """g ~ -4 (-12) per token: every cumulative decay factor underflows inside a chunk; the decay
+    differences are formed before the exponential, so nothing may overflow or turn into NaN."""
+    cfg = custom([300, 64, 700], 2, 4, seed=43, gate_mean=gate_mean)
+    check(cfg, "strong decay")
+    res = harness.run_prefill(cfg)
+    assert np.isfinite(res["out"]).all() and np.isfinite(res["final_state"]).all()

@@ -91,3 +91,17 @@ def test_split_prefill_repeated_calls_reuse_workspace():
     _, b = check(cfg, "second call")
     np.testing.assert_array_equal(a["out"], b["out"])
     np.testing.assert_array_equal(a["final_state"], b["final_state"])
+
+
+@pytest.mark.parametrize("gate_mean", [-4.0, -12.0])
+def test_split_prefill_strong_decay_underflows_cleanly(gate_mean):
+    """g ~ -4 (-12) per token: cumulative decays underflow to zero inside a chunk, the transition of a
+    run is exactly zero, and nothing may turn into NaN or Inf on the way."""
+    cfg = custom([1024], 4, 8, seed=37, gate_mean=gate_mean)
+    _, res = check(cfg, "strong decay, 4 runs")
+    assert np.isfinite(res["out"]).all() and np.isfinite(res["final_state"]).all()
+
+
+def test_split_prefill_long_ragged_sequence():
+    """20,001 tokens at 2/4 heads: 313 chunks in 8 runs of 40 (the last one 33 with a one-token tail)."""
+    check(custom([20001], 2, 4, seed=41, gate_mean=5.0), "long ragged sequence, 8 runs")
