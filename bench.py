@@ -336,16 +336,20 @@ def run_gpu(args):
         d_state, d_state_out = s_in[0], s_out[0]
         d_out16 = out.view(torch.int16)
 
+        # host buffers go through the package's pipelined host path (slices of the batch on three
+        # streams: both copy engines and the kernel busy at once); every byte still crosses PCIe each step
+        from paper_2607_16831_b200.host_pipeline import HostDecode
+
+        pipe = HostDecode(B, 16, 32, slices=8, streams=3)  # the state crosses PCIe: slice and overlap
+        pipe_res = HostDecode(B, 16, 32, slices=1, streams=1)  # the state stays on the device: one launch
+        pipe_res.s_in.copy_(d_state)
+
         def e2e_step(with_state):
-            for hsrc, ddst in zip(h_in, d_in):
-                ddst.copy_(hsrc, non_blocking=True)
             if with_state:
-                d_state.copy_(h_state, non_blocking=True)
-            gdn.gdn_decode(d_in[0].view(torch.bfloat16), d_in[1].view(torch.bfloat16), d_in[2].view(torch.bfloat16),
-                           d_in[3], d_in[4], d_state, d_state_out, out)
-            h_out.copy_(d_out16, non_blocking=True)
-            if with_state:
-                h_state_out.copy_(d_state_out, non_blocking=True)
+                pipe.step(h_in[0], h_in[1], h_in[2], h_in[3], h_in[4], h_state, h_state_out, h_out)
+            else:
+                pipe_res.step(h_in[0], h_in[1], h_in[2], h_in[3], h_in[4], None, None, h_out)
+                pipe_res.swap()
 
         def e2e_time(with_state, steps):
             for _ in range(3):
@@ -375,7 +379,9 @@ def run_gpu(args):
                            "h2d_bytes_per_step": tok_in + h_state.numel() * 4,
                            "d2h_bytes_per_step": h_out.numel() * 2 + h_state.numel() * 4,
                            "note": "every input (tokens and the 134 MB state) copied from pinned host memory and "
-                                   "every result copied back each step; PCIe-bound by construction"}
+                                   "every result copied back each step; PCIe-bound by construction. The batch moves "
+                                   "in 8 slices over 3 streams (host_pipeline.HostDecode) so that the copy in, the "
+                                   "kernel and the copy out overlap"}
             line["e2e_state_resident"] = {"value": world * B * STATE_BYTES_PER_ITEM / (ms_res * 1e-3) / 1e9,
                                           "unit": "GB/s", "ms_per_step": ms_res, "h2d_bytes_per_step": tok_in,
                                           "d2h_bytes_per_step": h_out.numel() * 2,

@@ -135,3 +135,33 @@ def test_decode_multi_token(B, T):
     got_o = harness.bf16_to_numpy(out).reshape(B * T, Hv, 128)
     e = harness.assert_close(got_o, ref_o, s_out.cpu().numpy().astype(np.float64), ref_s, "decode multi B=%d T=%d" % (B, T))
     assert e["state_rel_fro"] < 2e-6
+
+
+@pytest.mark.parametrize("B,slices,streams", [(5, 3, 2), (16, 8, 3), (2, 8, 3)])
+def test_decode_from_host_buffers_in_slices(B, slices, streams):
+    """host_pipeline.HostDecode: pinned host buffers in, slices of the batch on several streams,
+    pinned host buffers out; then a second step on the state kept on the device."""
+    import torch
+    from gdn_inputs import config
+    from paper_2607_16831_b200.host_pipeline import HostDecode
+
+    cfg = config("decode_sweep", B=B)
+    tok, st = cfg["tokens"], cfg["state"]
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    h = [pin(tok.q.view(np.int16)), pin(tok.k.view(np.int16)), pin(tok.v.view(np.int16)), pin(tok.g), pin(tok.beta)]
+    h_state = pin(st)
+    h_out = torch.full((B, tok.Hv, 128), -1, dtype=torch.int16).pin_memory()
+    h_state_out = torch.full_like(h_state, float("nan")).pin_memory()
+    pipe = HostDecode(B, tok.Hqk, tok.Hv, slices=slices, streams=streams)
+    pipe.step(*h, h_state, h_state_out, h_out)
+    torch.cuda.synchronize()
+    ref_o, ref_s = oracle.decode(*harness.token_arrays(tok), st)
+    got_o = harness.bf16_to_numpy(h_out.view(torch.bfloat16))
+    harness.assert_close(got_o, ref_o, h_state_out.numpy().astype(np.float64), ref_s, "host decode B=%d" % B)
+    # second step from the state that stayed on the device == oracle from the first step's state
+    pipe.swap()
+    pipe.step(*h, None, h_state_out, h_out)
+    torch.cuda.synchronize()
+    ref_o2, ref_s2 = oracle.decode(*harness.token_arrays(tok), ref_s.astype(np.float32))
+    harness.assert_close(harness.bf16_to_numpy(h_out.view(torch.bfloat16)), ref_o2,
+                         h_state_out.numpy().astype(np.float64), ref_s2, "host decode, second step")
