@@ -128,16 +128,16 @@ static cudaError_t launch(const void* q, const void* k, const void* v, const flo
                       (uint16_t*)out, Hqk, Hv, split);
 }
 
-// Launch-shape table.  `variant` < 0 picks from the batch size: below ~16 items the
-// kernel is latency bound and wants as many small CTAs as possible (one warp, four
-// rows: 1024 CTAs at B = 1); large batches want more bytes in flight per warp.
+// Launch-shape table.  `variant` < 0 picks from the number of (item, head) units; the other
+// shapes stay selectable for tuning on other head counts.
 cudaError_t decode_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
                             const float* A_log, const float* dt_bias, const float* s_in, float* s_out, void* out,
                             int B, int Hqk, int Hv, int variant, cudaStream_t st) {
     if (variant < 0) {
-        if (B <= 2) variant = 0;
-        else if (B <= 16) variant = 1;
-        else variant = 3;
+        // from sweeps of all variants at 8 and 32 value heads, B = 1 .. 512: four rows per warp in
+        // four-warp CTAs is the fastest shape from 16 (item, head) units upwards (3-7 % ahead of eight
+        // rows per warp: more, smaller CTAs keep more loads in flight); below that, one-warp CTAs
+        variant = ((long long)B * Hv <= 16) ? 0 : 8;
     }
     switch (variant) {
         case 0: return launch<1, 1>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
