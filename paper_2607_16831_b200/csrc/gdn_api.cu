@@ -158,7 +158,7 @@ int gdn_decode_variant(const void* q, const void* k, const void* v, const float*
                        stream);
 }
 
-int gdn_decode_num_variants(void) { return 10; }
+int gdn_decode_num_variants(void) { return 12; }
 
 int gdn_decode_multi(const void* q, const void* k, const void* v, const float* g, const float* beta,
                      const float* state_in, float* state_out, void* out, int B, int T, int Hqk, int Hv, int dk,

@@ -150,6 +150,8 @@ cudaError_t decode_dispatch(const void* q, const void* k, const void* v, const f
         case 7: return launch<8, 4>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
         case 8: return launch<1, 4>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
         case 9: return launch<2, 8>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
+        case 10: return launch<1, 2>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
+        case 11: return launch<1, 8>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, Hqk, Hv, st);
         default: return cudaErrorInvalidValue;
     }
 }
