@@ -36,7 +36,7 @@ PREFILL_FLOPS_PER_TOKEN = 5.77e6                         # 11.53 MFLOP per (chun
 # DRAM bytes per decode launch at B = 64 from the committed ncu capture
 # (profiles/decode_b64_ncu.md): 135.29 MB read + 79.69 MB written inside the launch window (the write-back
 # L2 still holds the tail of the 134 MB output when the kernel ends).
-DECODE_B64_DRAM_TRAFFIC = 219.41e6
+DECODE_B64_DRAM_TRAFFIC = 218.03e6
 
 
 def load_peaks():
