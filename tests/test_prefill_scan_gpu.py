@@ -43,6 +43,9 @@ SHAPES = [
     ([1100], 8, 16, "18 chunks, 16 heads -> 4 runs (5,5,5,3)"),
     ([1500, 700], 4, 8, "two sequences -> 5 runs each; the short one has runs of 3, 3, 3, 2, 0 chunks"),
     ([900, 0, 64], 2, 4, "an empty sequence and a one-chunk sequence beside a split one"),
+    ([1024], 8, 8, "one value head per key head"),
+    ([1024], 2, 8, "four value heads per key head"),
+    ([1024], 1, 3, "three value heads on one key head (an unpaired head in the intra-chunk kernel)"),
 ]
 
 
