@@ -18,10 +18,16 @@
 // arrive by TMA from the caller's tensors, the chunk summaries by bulk copies of
 // pre-swizzled images, two stages deep.  The fp32 state stays in tensor memory for the
 // whole sequence.  Warp roles:
-//   warps 0-3  chain: drain Delta^T -> bf16 operands; drain S -> bf16 operand + decayed fp32 back
-//   warps 4-7  output: drain Oa/Ob -> bf16 out
-//   warp  8    issues every MMA (one elected lane)
-//   warp  9    issues every TMA / bulk copy, one chunk ahead of the MMAs
+//   warp  0     issues every MMA (one elected lane)
+//   warp  1     issues every TMA / bulk copy, one chunk ahead of the MMAs
+//   warps 4-7   chain: drain Delta^T -> bf16 operands; drain S -> bf16 operand + decayed fp32 back
+//   warps 8-11  output: drain Oa/Ob -> bf16 out
+//   (warps 2, 3 idle: a role that touches tensor memory needs warp % 4 = its lane quarter)
+// Measured with clock stamps: tcgen05.ld / tcgen05.st of one warp queue behind MMAs that are already
+// in flight (the drain of Delta^T takes ~590 clocks with an empty MMA queue and ~890 with the eight
+// S Q^T MMAs queued in front of it), so every off-chain product lengthens the chain by about its own
+// duration wherever it is issued; only the ~200-clock gaps between an MMA's completion and the
+// waiting warp seeing its mbarrier are free.
 // Hand-offs are mbarriers; every wait is bounded and failure unwinds through an abort flag.
 //
 // With `segs` > 1 a sequence is cut into that many runs of chunks and the runs advance at the same
@@ -36,7 +42,8 @@
 namespace gdn {
 using namespace sm100;
 
-constexpr int kChainThreads = 320;
+constexpr int kChainThreads = 384;
+constexpr int kIssuerWarp = 0, kProducerWarp = 1, kChainWarp0 = 4, kOutputWarp0 = 8;  // warps 2, 3 idle
 
 // One arrival per warp: 128 threads arriving on the same mbarrier are serialised by the
 // shared-memory unit (~500 clk before the waiter sees the phase complete); the lanes are ordered
@@ -70,7 +77,7 @@ constexpr uint32_t TM_DTH = 416;    // bf16 (e o Delta)^T hi          32
 constexpr uint32_t TM_DTL = 448;    // bf16 (e o Delta)^T lo          32
 constexpr uint32_t TM_COLS = 512;
 
-enum { B_FULL_A0 = 0, B_FULL_A1, B_FULL_B0, B_FULL_B1, B_FREE0, B_FREE1, B_DELTA, B_STATE, B_O, B_DW, B_SHI, B_STM, B_OFREE, B_COUNT };
+enum { B_FULL_A0 = 0, B_FULL_A1, B_FULL_B0, B_FULL_B1, B_FREE0, B_FREE1, B_DELTA, B_STATE, B_O, B_DW, B_SHI, B_STM, B_OFREE, B_DL, B_COUNT };
 
 __global__ void __launch_bounds__(kChainThreads, 1)
 gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -138,13 +145,13 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
     if (tid == 0) {
         for (int i = 0; i < B_COUNT; ++i) {
-            const bool many = (i == B_DW || i == B_SHI || i == B_STM || i == B_OFREE);
+            const bool many = (i == B_DW || i == B_SHI || i == B_STM || i == B_OFREE || i == B_DL);
             mbar_init(bars + i, many ? 4u : 1u);  // one arrival per warp of the arriving role
         }
         *abort_flag = 0;
         mbar_fence_init();
     }
-    if (warp == 8) {
+    if (warp == kIssuerWarp) {
         __syncwarp();
         tmem_alloc(tmem_slot, TM_COLS);
     }
@@ -158,7 +165,8 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     };
 #ifdef GDN_CHAIN_PROFILE
     // SM-clock stamps of CTA 0 into the unused tail of each chunk's scalar block (4-byte slots from byte 576)
-#define GDN_STAMP(c, slot) do { if (blockIdx.x == 0) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)(c) * Hv + h) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
+// GDN_CHAIN_PROFILE is a bit mask of the stamp slots to record (every stamp costs its warp ~150 clocks)
+#define GDN_STAMP(c, slot) do { if ((((unsigned long long)(GDN_CHAIN_PROFILE) >> (slot)) & 1ull) && blockIdx.x == 0) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)(c) * Hv + h) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
 #else
 #define GDN_STAMP(c, slot) do { } while (0)
 #endif
@@ -168,7 +176,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)c_begin * Hv + h) * kScalBytes + 576)[43] = t_entry;
 #endif
 
-    if (warp == 8) {
+    if (warp == kIssuerWarp) {
         // =========================================================== issuer: MMA
         // The whole warp runs this loop in lock step; one elected lane issues each MMA.  Values that
         // feed the MMA operands are broadcast from lane 0 so that the compiler knows they are
@@ -204,6 +212,8 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             bool g1_issued = false;
 
 #define GDN_WAIT(idx, parity) if (!mbar_wait_all(bars + (idx), (uint32_t)(parity), abort_flag)) break
+// for barriers that have normally completed long before the issuer gets here
+#define GDN_WAIT_READY(idx, parity) if (!mbar_wait_all_probe(bars + (idx), (uint32_t)(parity), abort_flag)) break
 
             for (int ci = 0; ci < nchunks_u; ++ci) {
                 const int c = c_begin + ci;
@@ -233,8 +243,11 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
                 umma_commit_warp(bars + B_DELTA);
                 if (lane == 0) GDN_STAMP(c, 4);
-                // ---- off the chain: Oa^T = S Q^T (runs while the chain warps drain Delta^T)
-                if (ci >= 1) GDN_WAIT(B_OFREE, par ^ 1);
+                // ---- off the chain: Oa^T = S Q^T (runs while the chain warps drain Delta^T).  The waits
+                //      that G3B needs besides Delta are taken here, where nobody is waiting for the issuer
+                if (ci >= 1) GDN_WAIT_READY(B_OFREE, par ^ 1);
+                GDN_WAIT_READY(B_FULL_B0 + st, ph2);
+                GDN_WAIT_READY(B_STM, par);
                 {
                     const uint64_t q0 = dQ0 + so, q1 = dQ1 + so;
                     const uint32_t td = tmem_base_u + TM_OA, ta = tmem_base_u + TM_SHI;
@@ -245,8 +258,6 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
                 if (lane == 0) GDN_STAMP(c, 5);
                 // ---- on the chain: S += (e o Delta)^T K  (hi + lo; A in tensor memory, B = K MN-major)
-                GDN_WAIT(B_FULL_B0 + st, ph2);
-                GDN_WAIT(B_STM, par);
                 if (lane == 0) GDN_STAMP(c, 7);
                 GDN_WAIT(B_DW, par);
                 if (lane == 0) GDN_STAMP(c, 8);
@@ -262,11 +273,13 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 umma_commit_warp(bars + B_STATE);
                 if (lane == 0) GDN_STAMP(c, 9);
                 // ---- off the chain: Ob^T = Delta^T P^T, and the next chunk's V^T T'^T if it has landed
+                GDN_WAIT(B_DL, par);
+                tc_fence_after_sync();
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
                     umma_bf16_ts_warp(tmem_base_u + TM_OB, tmem_base_u + TM_DL + ks * 8, dP + so + ks * 2, ID_N64, ks > 0);
                 if (!last) {
-                    GDN_WAIT(B_FULL_A0 + (st ^ 1), ((ci + 1) >> 1) & 1);  // requested a whole chunk ago
+                    GDN_WAIT_READY(B_FULL_A0 + (st ^ 1), ((ci + 1) >> 1) & 1);  // requested a whole chunk ago
                     tc_fence_after_sync();
                     if (!ident_u) issue_G1(st ^ 1);
                     g1_issued = true;
@@ -276,9 +289,10 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 if (lane == 0) GDN_STAMP(c, 10);
             }
 #undef GDN_WAIT
+#undef GDN_WAIT_READY
         }
         __syncwarp();
-    } else if (warp == 9) {
+    } else if (warp == kProducerWarp) {
         // =========================================================== producer: all TMA / bulk copies
         {
             if (lane == 0) {
@@ -311,10 +325,10 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
         }
         __syncwarp();
-    } else if (warp < 4) {
+    } else if (warp >= kChainWarp0 && warp < kChainWarp0 + 4) {
         // =========================================================== chain warps
-        const int v = tid;
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
+        const int v = tid - kChainWarp0 * 32;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
         const size_t sbase = (size_t)v * kD;
         // initial state: bf16 operand copy and Gamma_L(first chunk) * S, both into tensor memory
         {
@@ -356,7 +370,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tc_fence_before_sync();
             warp_arrive(bars + B_SHI);
             warp_arrive(bars + B_STM);
-            if (tid == 0) GDN_STAMP(c_begin, 42);  // initial state in tensor memory
+            if (tid == kChainWarp0 * 32) GDN_STAMP(c_begin, 42);  // initial state in tensor memory
         }
         for (int ci = 0; ci < nchunks; ++ci) {
             const int c = c_begin + ci;
@@ -371,38 +385,52 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 for (int j = 0; j < 16; ++j) ev4[j] = __ldg(e4 + j);
                 if (!last) asm volatile("prefetch.global.L2 [%0];" ::"l"(scal_ptr(c + 1) + (lane & 3) * 32));
             }
-            if (tid == 0) GDN_STAMP(c, 16);
+            if (tid == kChainWarp0 * 32) GDN_STAMP(c, 16);
             if (!mbar_wait_all(bars + B_DELTA, par, abort_flag)) break;
             tc_fence_after_sync();
-            if (tid == 0) GDN_STAMP(c, 17);
-            // Delta^T row v -> bf16 A operands in tensor memory: Delta, and (e o Delta) as hi + lo.
-            // Two halves of 32 tokens keep the live registers low (9 warps share the register file).
+            if (tid == kChainWarp0 * 32) GDN_STAMP(c, 17);
+            // Delta^T row v -> bf16 A operands in tensor memory.  First (e o Delta) as hi + lo, which
+            // the state update on the chain is waiting for; the plain bf16 Delta that only the output
+            // product needs follows after that hand-off.  Two halves of 32 tokens keep the live
+            // registers low (the warps share the register file).
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                uint32_t r[32], xd[16], hd[16], ld[16];
+                uint32_t r[32], hd[16], ld[16];
                 tmem_ld32(lane_addr + TM_DELTA + half * 32, r);
                 tmem_ld_wait();
-                if (tid == 0 && half == 0) GDN_STAMP(c, 28);
+                if (tid == kChainWarp0 * 32 && half == 0) GDN_STAMP(c, 28);
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     const float4 ea = ev4[half * 8 + (j >> 1)];
                     const float e0 = (j & 1) ? ea.z : ea.x, e1 = (j & 1) ? ea.w : ea.y;
-                    const float x0 = __uint_as_float(r[2 * j]), x1 = __uint_as_float(r[2 * j + 1]);
-                    xd[j] = pack_bf16x2(x0, x1);
-                    split_bf16x2(x0 * e0, x1 * e1, hd[j], ld[j]);
+                    split_bf16x2(__uint_as_float(r[2 * j]) * e0, __uint_as_float(r[2 * j + 1]) * e1, hd[j], ld[j]);
                 }
                 tmem_st16(lane_addr + TM_DTH + half * 16, hd);
                 tmem_st16(lane_addr + TM_DTL + half * 16, ld);
-                tmem_st16(lane_addr + TM_DL + half * 16, xd);
             }
             tmem_st_wait();
             tc_fence_before_sync();
             warp_arrive(bars + B_DW);
-            if (tid == 0) GDN_STAMP(c, 18);
+            if (tid == kChainWarp0 * 32) GDN_STAMP(c, 18);
+            {   // off the chain: bf16 Delta^T for Ob^T = Delta^T P^T (the accumulator is intact until
+                // the next chunk's V^T T'^T, which the issuer starts only after this hand-off)
+                uint32_t r[32], xd[32];
+                tmem_ld32(lane_addr + TM_DELTA, r);
+                tmem_ld32(lane_addr + TM_DELTA + 32, xd);  // second half, packed in place below
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) r[j] = pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+#pragma unroll
+                for (int j = 0; j < 16; ++j) r[16 + j] = pack_bf16x2(__uint_as_float(xd[2 * j]), __uint_as_float(xd[2 * j + 1]));
+                tmem_st32(lane_addr + TM_DL, r);
+                tmem_st_wait();
+                tc_fence_before_sync();
+                warp_arrive(bars + B_DL);
+            }
 
             if (!mbar_wait_all(bars + B_STATE, par, abort_flag)) break;
             tc_fence_after_sync();
-            if (tid == 0) GDN_STAMP(c, 19);
+            if (tid == kChainWarp0 * 32) GDN_STAMP(c, 19);
             if (last) {
                 if (fin_ptr) {
                     // run 0 of a split sequence also leaves its final state as the bf16 operand tiles
@@ -446,7 +474,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 tmem_st_wait();
                 tc_fence_before_sync();
                 warp_arrive(bars + B_SHI);
-                if (tid == 0) GDN_STAMP(c, 20);
+                if (tid == kChainWarp0 * 32) GDN_STAMP(c, 20);
                 // ... then the fp32 state decayed by the next chunk's Gamma_L, in place (gates the next G3B)
 #pragma unroll
                 for (int b = 0; b < 2; ++b) {
@@ -465,12 +493,12 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 tmem_st_wait();
                 tc_fence_before_sync();
                 warp_arrive(bars + B_STM);
-                if (tid == 0) GDN_STAMP(c, 21);
+                if (tid == kChainWarp0 * 32) GDN_STAMP(c, 21);
             }
         }
-    } else {
+    } else if (warp >= kOutputWarp0) {
         // =========================================================== output warps
-        const int v = tid - 128;
+        const int v = tid - kOutputWarp0 * 32;
         const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
         for (int ci = 0; ci < nchunks; ++ci) {
             const int c = c_begin + ci;
@@ -479,10 +507,10 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             auto last_chunk = [&](int i) { return i + 1 == nchunks; };
             const float4* g4 = reinterpret_cast<const float4*>(scal_ptr(c));  // Gamma_i of this chunk
             if (!last_chunk(ci)) asm volatile("prefetch.global.L2 [%0];" ::"l"(scal_ptr(c + 1) + (lane & 1) * 32));
-            if (tid == 128) GDN_STAMP(c, 24);
+            if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 24);
             if (!mbar_wait_all(bars + B_O, par, abort_flag)) break;
             tc_fence_after_sync();
-            if (tid == 128) GDN_STAMP(c, 25);
+            if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 25);
             // drain both accumulators into registers and hand the columns back at once: the next
             // chunk's S Q^T is waiting for them
             uint32_t a0[32], a1[32], b0[32], b1[32];
@@ -493,7 +521,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tmem_ld_wait();
             tc_fence_before_sync();
             warp_arrive(bars + B_OFREE);
-            if (tid == 128) GDN_STAMP(c, 26);
+            if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 26);
             // o_i = Gamma_i Oa^T[v][i] + Ob^T[v][i], packed two tokens per register
             uint32_t op[32];
 #pragma unroll
@@ -532,7 +560,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                             *reinterpret_cast<const uint4*>(ost + row * kD + c16 * 8);
                 }
             }
-            if (tid == 128) GDN_STAMP(c, 27);
+            if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 27);
         }
     }
 
@@ -545,7 +573,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 8) {
+    if (warp == kIssuerWarp) {
         __syncwarp();
         tmem_dealloc(tmem_base, TM_COLS);
     }

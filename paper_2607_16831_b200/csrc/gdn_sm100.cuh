@@ -99,6 +99,25 @@ __device__ __forceinline__ bool mbar_wait_all(uint64_t* bar, uint32_t parity, vo
                                               long long limit_cycles = 2000000000LL) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort, limit_cycles));
 }
+// Non-blocking check of a phase (mbarrier.test_wait never suspends the thread).
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// For waits that are usually satisfied already: one non-blocking test by every lane (~18 clocks for
+// a completed phase against ~60 for try_wait); falls back to mbar_wait_all when the phase is open.
+__device__ __forceinline__ bool mbar_wait_all_probe(uint64_t* bar, uint32_t parity, volatile int* abort,
+                                                    long long limit_cycles = 2000000000LL) {
+    if (__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) return true;
+    return mbar_wait_all(bar, parity, abort, limit_cycles);
+}
 
 // ---------------------------------------------------------------- fences
 __device__ __forceinline__ void fence_proxy_async_smem() {
