@@ -23,11 +23,11 @@
 //   warps 4-7   chain: drain Delta^T -> bf16 operands; drain S -> bf16 operand + decayed fp32 back
 //   warps 8-11  output: drain Oa/Ob -> bf16 out
 //   (warps 2, 3 idle: a role that touches tensor memory needs warp % 4 = its lane quarter)
-// Measured with clock stamps: tcgen05.ld / tcgen05.st of one warp queue behind MMAs that are already
-// in flight (the drain of Delta^T takes ~590 clocks with an empty MMA queue and ~890 with the eight
-// S Q^T MMAs queued in front of it), so every off-chain product lengthens the chain by about its own
-// duration wherever it is issued; only the ~200-clock gaps between an MMA's completion and the
-// waiting warp seeing its mbarrier are free.
+// Measured with clock stamps (GDN_CHAIN_PROFILE): a chunk step is ~3150 clocks and stays there when the
+// off-chain products are moved around; the drain of Delta^T takes ~590 clocks when no other MMA is issued or
+// executing at the time and 100-300 more when the eight S Q^T MMAs are (in a microbenchmark queued MMAs do
+// not delay another warp's tcgen05.ld / st at all, so this is contention inside the kernel, part of it the
+// issuer sharing a scheduler with chain warp 0).
 // Hand-offs are mbarriers; every wait is bounded and failure unwinds through an abort flag.
 //
 // With `segs` > 1 a sequence is cut into that many runs of chunks and the runs advance at the same
@@ -243,11 +243,8 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
                 umma_commit_warp(bars + B_DELTA);
                 if (lane == 0) GDN_STAMP(c, 4);
-                // ---- off the chain: Oa^T = S Q^T (runs while the chain warps drain Delta^T).  The waits
-                //      that G3B needs besides Delta are taken here, where nobody is waiting for the issuer
+                // ---- off the chain: Oa^T = S Q^T (executes while the chain warps drain Delta^T)
                 if (ci >= 1) GDN_WAIT_READY(B_OFREE, par ^ 1);
-                GDN_WAIT_READY(B_FULL_B0 + st, ph2);
-                GDN_WAIT_READY(B_STM, par);
                 {
                     const uint64_t q0 = dQ0 + so, q1 = dQ1 + so;
                     const uint32_t td = tmem_base_u + TM_OA, ta = tmem_base_u + TM_SHI;
@@ -258,6 +255,8 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
                 if (lane == 0) GDN_STAMP(c, 5);
                 // ---- on the chain: S += (e o Delta)^T K  (hi + lo; A in tensor memory, B = K MN-major)
+                GDN_WAIT_READY(B_FULL_B0 + st, ph2);
+                GDN_WAIT_READY(B_STM, par);
                 if (lane == 0) GDN_STAMP(c, 7);
                 GDN_WAIT(B_DW, par);
                 if (lane == 0) GDN_STAMP(c, 8);
@@ -278,13 +277,15 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
                     umma_bf16_ts_warp(tmem_base_u + TM_OB, tmem_base_u + TM_DL + ks * 8, dP + so + ks * 2, ID_N64, ks > 0);
+                // both output accumulators are complete with this product: the output warps can drain them
+                // (and hand Oa^T back for the next chunk's S Q^T) without waiting for V^T T'^T as well
+                umma_commit_warp(bars + B_O);
                 if (!last) {
                     GDN_WAIT_READY(B_FULL_A0 + (st ^ 1), ((ci + 1) >> 1) & 1);  // requested a whole chunk ago
                     tc_fence_after_sync();
                     if (!ident_u) issue_G1(st ^ 1);
                     g1_issued = true;
                 }
-                umma_commit_warp(bars + B_O);
                 umma_commit_warp(bars + B_FREE0 + st);  // every MMA that reads this stage has been issued
                 if (lane == 0) GDN_STAMP(c, 10);
             }
@@ -389,6 +390,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             if (!mbar_wait_all(bars + B_DELTA, par, abort_flag)) break;
             tc_fence_after_sync();
             if (tid == kChainWarp0 * 32) GDN_STAMP(c, 17);
+            if (lane == 0) GDN_STAMP(c, 36 + (warp & 3));
             // Delta^T row v -> bf16 A operands in tensor memory.  First (e o Delta) as hi + lo, which
             // the state update on the chain is waiting for; the plain bf16 Delta that only the output
             // product needs follows after that hand-off.  Two halves of 32 tokens keep the live
@@ -412,6 +414,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tc_fence_before_sync();
             warp_arrive(bars + B_DW);
             if (tid == kChainWarp0 * 32) GDN_STAMP(c, 18);
+            if (lane == 0) GDN_STAMP(c, 32 + (warp & 3));
             {   // off the chain: bf16 Delta^T for Ob^T = Delta^T P^T (the accumulator is intact until
                 // the next chunk's V^T T'^T, which the issuer starts only after this hand-off)
                 uint32_t r[32], xd[32];
