@@ -396,8 +396,12 @@ def run_gpu(args):
             med, mn = time_graph(lambda i: gdn.gdn_decode(ds["q"], ds["k"], ds["v"], ds["g"], ds["beta"], si[i % nb],
                                                           so[i % nb], oo), iters=40)
             gbs = Bs * STATE_BYTES_PER_ITEM / med / 1e3
+            # warm: the same pair of state buffers every call (the 126 MB L2 holds them up to B ~ 16)
+            warm, _ = time_graph(lambda i: gdn.gdn_decode(ds["q"], ds["k"], ds["v"], ds["g"], ds["beta"], si[0], so[0], oo),
+                                 iters=40)
             sweep.append({"B": Bs, "us_per_call": med, "us_min": mn, "state_gbs": gbs, "frac_measured": gbs / peaks["hbm"],
-                          "frac_8TBs": gbs / 8000.0, "regime": "latency-bound" if Bs < 8 else "bandwidth-bound"})
+                          "frac_8TBs": gbs / 8000.0, "us_per_call_warm_same_buffers": warm,
+                          "regime": "latency-bound" if Bs < 8 else "bandwidth-bound"})
             del cfg_s, ds, si, so, oo
             torch.cuda.empty_cache()
         line["decode_sweep"] = {"timing": "40 back-to-back calls in one CUDA graph, cold (rotating) state buffers",
@@ -451,9 +455,15 @@ def run_gpu(args):
         pre.append(dict(bench_prefill("short", peaks, reps, lengths=[8] * 64, Hqk=4, Hv=8,
                                       env={"GDN_PREFILL_SHORT_FALLBACK": "0"}),
                         variant="4/8 heads, 64 sequences of 8 tokens, chunked kernels forced"))
+        # µs per chunk step of the serial chain: one sequence of 4096 tokens against two of 2048 (the same
+        # intra-chunk work, 32 more dependent steps), sequence split switched off
+        off = {"GDN_PREFILL_MAX_SEGMENTS": "1"}
+        t64 = bench_prefill("one", peaks, reps, lengths=[4096], env=off)["us"]
+        t32 = bench_prefill("two", peaks, reps, lengths=[2048, 2048], env=off)["us"]
         line["prefill"] = {"rooflines": {"hbm_gbs": peaks["hbm"], "bf16_tflops": peaks["bf16"], "source": peaks["source"],
                                          "bytes_per_token": PREFILL_BYTES_PER_TOKEN,
-                                         "flops_per_token": PREFILL_FLOPS_PER_TOKEN}, "runs": pre}
+                                         "flops_per_token": PREFILL_FLOPS_PER_TOKEN},
+                           "chain_us_per_chunk_step": (t64 - t32) / 32.0, "runs": pre}
         # ---- CPU oracle on this machine's host cores (reported baseline, not the target)
         import oracle
 
