@@ -164,10 +164,11 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int hq = blockIdx.y / npairs, p = blockIdx.y % npairs;
 #ifdef GDN_INTRA_PROFILE
     // SM-clock stamps of thread 0 into the unused tail of this CTA's first scalar block (4-byte slots from byte 576)
-#define GDN_ISTAMP(slot) do { if (threadIdx.x == 0) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)c * Hv + hq * G + 2 * p) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
+#define GDN_ISTAMP_T(thread, slot) do { if (threadIdx.x == (thread)) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)c * Hv + hq * G + 2 * p) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
 #else
-#define GDN_ISTAMP(slot) do { } while (0)
+#define GDN_ISTAMP_T(thread, slot) do { } while (0)
 #endif
+#define GDN_ISTAMP(slot) GDN_ISTAMP_T(0, slot)
     GDN_ISTAMP(0);
     const int hh = tid >> 6, i = tid & 63;  // role in the gate / solve / W phases: head of the pair, row
     const int nh = min(2, G - 2 * p);
@@ -286,6 +287,9 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             const int jb_own = row >> 4;
 #pragma unroll 1
             for (int q4 = 0; q4 < 4; ++q4) {
+                GDN_ISTAMP_T(0, 14 + q4);    // P side (warp 0)
+                GDN_ISTAMP_T(64, 20 + q4);   // A side (warp 2)
+                GDN_ISTAMP_T(96, 26 + q4);   // A side (warp 3)
                 uint32_t r[16];
                 tmem_ld16(lane_addr + ITM_D1 + q4 * 16, r);
                 tmem_ld_wait();
@@ -305,8 +309,12 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                             for (int jl = 0; jl < 16; ++jl) pv[jl] = __uint_as_float(r[jl]) * (rf * cf[jl]);
                         } else if (q4 == jb_own && row < len) {  // the diagonal block
 #pragma unroll
-                            for (int jl = 0; jl < 16; ++jl)
-                                pv[jl] = (q4 * 16 + jl <= row) ? __uint_as_float(r[jl]) * __expf(gi - gm[jl]) : 0.f;
+                            for (int jl = 0; jl < 16; ++jl) {
+                                // exponent clamped instead of masked: no branch per element (the masked
+                                // elements, where it would be positive, are zeroed by the select)
+                                const float d = __expf(fminf(gi - gm[jl], 0.f));
+                                pv[jl] = (q4 * 16 + jl <= row) ? __uint_as_float(r[jl]) * d : 0.f;
+                            }
                         } else {
 #pragma unroll
                             for (int jl = 0; jl < 16; ++jl) pv[jl] = 0.f;
@@ -323,8 +331,10 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         if (q4 == jb_own) {
                             const float* bm = bet + e * 64 + q4 * 16;
 #pragma unroll
-                            for (int ml = 0; ml < 16; ++ml)
-                                a[ml] = (q4 * 16 + ml > row) ? bm[ml] * __expf(gm[ml] - gi) * __uint_as_float(r[ml]) : 0.f;
+                            for (int ml = 0; ml < 16; ++ml) {
+                                const float d = bm[ml] * __expf(fminf(gm[ml] - gi, 0.f));
+                                a[ml] = (q4 * 16 + ml > row) ? d * __uint_as_float(r[ml]) : 0.f;
+                            }
                         } else {
                             const float rf = __expf(gam[e * 64 + q4 * 16] - gi);
                             const float* cf = cfA + e * 64 + q4 * 16;
@@ -352,6 +362,9 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
             }
         }
+        GDN_ISTAMP_T(0, 18);
+        GDN_ISTAMP_T(64, 24);
+        GDN_ISTAMP_T(96, 30);
         fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncthreads();  // B tiles and diagonal blocks complete; the accumulator of MMA1 is dead from here on
