@@ -89,8 +89,8 @@ constexpr uint32_t IDG = IQ_LO;    // after MMA1: diagonal blocks of A^T, fp32 [
 constexpr uint32_t IBT2 = IQ_HI;   // after MMA1: B tiles of column block 2 (hi 4 KB | lo 4 KB)
 constexpr uint32_t IBT = 32768;    // B tiles of column blocks 0 and 1: [jb][hi|lo] x 4 KB               16 KB
 constexpr uint32_t IT2 = IBT;      // after the solve: T'' operand (bf16) [128][64]                       16 KB
-constexpr uint32_t IGAM = IBT + 16384;  // gam[2][64] | bet[2][64] | Gam[2][64] | cfP[2][64] | cfA[2][64] | tmp[4]
-constexpr uint32_t IBAR = IGAM + 10 * 64 * 4 + 64;
+constexpr uint32_t IGAM = IBT + 16384;  // gam[2][64] | bet[2][64] | Gam[2][64] | cfP[2][64] | cfA[2][64] | alp[2][64] | tmp[4]
+constexpr uint32_t IBAR = IGAM + 12 * 64 * 4 + 64;
 constexpr uint32_t kIntraSmem = IBAR + 64 + 1024;
 // tensor-memory columns: [QK^T ; KK^T] first, then the solve's operands, then the W accumulator
 constexpr uint32_t ITM_D1 = 0, ITM_YHI = 0, ITM_YLO = 32, ITM_ACC = 64, ITM_D2 = 0, ITM_COLS = 128;
@@ -182,7 +182,8 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     float* Gam = gam + 256;
     float* cfP = gam + 384;  // exp(gamma_{last column of j's 16-block} - gamma_j)
     float* cfA = gam + 512;  // beta_m exp(gamma_m - gamma_{first row of m's 16-block})
-    float* tmp = gam + 640;
+    float* alp = gam + 640;  // per-token decay exp(g_t) = exp(gamma_t - gamma_{t-1})
+    float* tmp = gam + 768;
     uint64_t* bar_load = reinterpret_cast<uint64_t*>(smem + IBAR);
     uint64_t* bar_mma1 = bar_load + 1;
     uint64_t* bar_mma2 = bar_load + 2;
@@ -232,6 +233,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             // with A_log given, g/beta are the raw gate inputs a and b
             if (A_log) raw_gates(x, b, __ldg(A_log + h), __ldg(dt_bias + h), x, b);
         }
+        alp[tid] = __expf(x);
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const float y = __shfl_up_sync(0xffffffffu, x, o);
@@ -302,18 +304,26 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         // P row: (Q K^T)_ij exp(gamma_i - gamma_j) for j <= i (difference masked before exp)
                         uint8_t* wsP = ws + L.off_P + ((size_t)c * Hv + hq * G + 2 * p + e) * kPBytes;
                         float pv[16];
-                        if (q4 < jb_own && row < len) {        // whole block left of the diagonal block
-                            const float rf = __expf(gi - gam[e * 64 + q4 * 16 + 15]);
+                        // Branch conditions are uniform over the warp (its 32 rows span two 16-blocks):
+                        // column blocks left of both use the factored decay; the two blocks that hold a
+                        // diagonal block for one half of the warp take the per-element form for all 32 lanes.
+                        const int wb2 = (row >> 5) * 2;
+                        if (q4 < wb2) {
+                            const float rf = (row < len) ? __expf(gi - gam[e * 64 + q4 * 16 + 15]) : 0.f;
                             const float* cf = cfP + e * 64 + q4 * 16;
 #pragma unroll
                             for (int jl = 0; jl < 16; ++jl) pv[jl] = __uint_as_float(r[jl]) * (rf * cf[jl]);
-                        } else if (q4 == jb_own && row < len) {  // the diagonal block
+                        } else if (q4 <= wb2 + 1) {
+                            // exp(gamma_i - gamma_j) from the right end of the block by a running product
+                            // of the per-token decays (one exp per row instead of sixteen; every factor
+                            // is <= 1, so nothing can overflow): acc = exp(gamma_i - gamma_j) once j <= i
+                            float acc = __expf(fminf(gi - gm[15], 0.f));  // 1 for rows inside the block
+                            const float* al = alp + e * 64 + q4 * 16;
 #pragma unroll
-                            for (int jl = 0; jl < 16; ++jl) {
-                                // exponent clamped instead of masked: no branch per element (the masked
-                                // elements, where it would be positive, are zeroed by the select)
-                                const float d = __expf(fminf(gi - gm[jl], 0.f));
-                                pv[jl] = (q4 * 16 + jl <= row) ? __uint_as_float(r[jl]) * d : 0.f;
+                            for (int jl = 15; jl >= 0; --jl) {
+                                const bool on = (q4 * 16 + jl <= row) && (row < len);
+                                pv[jl] = on ? __uint_as_float(r[jl]) * acc : 0.f;
+                                acc = on ? acc * al[jl] : acc;
                             }
                         } else {
 #pragma unroll
@@ -330,10 +340,14 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         float a[16];
                         if (q4 == jb_own) {
                             const float* bm = bet + e * 64 + q4 * 16;
+                            // exp(gamma_m - gamma_j), m > j, as the running product of the per-token decays
+                            const float* al = alp + e * 64 + q4 * 16;
+                            float acc = 1.f;
 #pragma unroll
                             for (int ml = 0; ml < 16; ++ml) {
-                                const float d = bm[ml] * __expf(fminf(gm[ml] - gi, 0.f));
-                                a[ml] = (q4 * 16 + ml > row) ? d * __uint_as_float(r[ml]) : 0.f;
+                                const bool on = q4 * 16 + ml > row;
+                                acc = on ? acc * al[ml] : acc;
+                                a[ml] = on ? bm[ml] * acc * __uint_as_float(r[ml]) : 0.f;
                             }
                         } else {
                             const float rf = __expf(gam[e * 64 + q4 * 16] - gi);
