@@ -543,6 +543,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             // 256-byte rows per half warp (64 two-byte stores per thread kept these warps busier than
             // the chain itself).  The named barrier covers the four output warps only; every one of
             // them reaches it in every iteration.
+            if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 44);
             {
                 uint16_t* ost = reinterpret_cast<uint16_t*>(smem + OFF_OST);
                 asm volatile("bar.sync 1, 128;" ::: "memory");  // the previous chunk's tile has been read
@@ -551,7 +552,9 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     ost[(2 * j) * kD + v] = (uint16_t)(op[j] & 0xffffu);
                     ost[(2 * j + 1) * kD + v] = (uint16_t)(op[j] >> 16);
                 }
+                if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 45);
                 asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 46);
                 const int c16 = v & 15, r0 = v >> 4;
                 uint16_t* obase = out_ptr + ((size_t)t0 * Hv + h) * kD + c16 * 8;
                 const size_t ostride = (size_t)Hv * kD;
