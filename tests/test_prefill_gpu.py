@@ -182,3 +182,65 @@ def test_prefill_strong_decay_underflows_cleanly(gate_mean):
     check(cfg, "strong decay")
     res = harness.run_prefill(cfg)
     assert np.isfinite(res["out"]).all() and np.isfinite(res["final_state"]).all()
+
+
+def test_prefill_all_sequences_empty_passes_states_through():
+    from gdn_inputs import Tokens
+    N, Hqk, Hv = 3, 2, 4
+    empty = Tokens(q=np.zeros((0, Hqk, 128), np.uint16), k=np.zeros((0, Hqk, 128), np.uint16),
+                   v=np.zeros((0, Hv, 128), np.uint16), g=np.zeros((0, Hv), np.float32),
+                   beta=np.zeros((0, Hv), np.float32), Hqk=Hqk, Hv=Hv, dk=128, dv=128)
+    init = make_state(N, Hv, seed=47)
+    res = harness.run_prefill(dict(tokens=empty, cu_seqlens=make_cu_seqlens([0] * N), initial_state=init))
+    np.testing.assert_array_equal(res["final_state"], init.astype(np.float64))
+    res = harness.run_prefill(dict(tokens=empty, cu_seqlens=make_cu_seqlens([0] * N), initial_state=None))
+    assert np.count_nonzero(res["final_state"]) == 0
+
+
+def test_prefill_beta_zero_is_pure_decay_closed_form():
+    """beta = 0: nothing is written, S_T = exp(sum g) S_0 and o_t = exp(gamma_t) S_0 q_t -- checked
+    against that closed form in fp64, not against the oracle (T = 300 spans five chunks)."""
+    from gdn_inputs import bf16_bits_to_f32
+    T, Hqk, Hv = 300, 2, 4
+    tok = make_tokens(T, Hqk, Hv, seed=53, gate_mean=4.0)
+    tok.beta[:] = 0.0
+    init = make_state(1, Hv, seed=53)
+    res = harness.run_prefill(dict(tokens=tok, cu_seqlens=make_cu_seqlens([T]), initial_state=init))
+    q = bf16_bits_to_f32(tok.q).astype(np.float64)
+    gam = np.cumsum(tok.g.astype(np.float64), axis=0)  # [T, Hv]
+    S0 = init[0].astype(np.float64)                    # [Hv, dv, dk]
+    ref_o = np.stack([np.exp(gam[:, h])[:, None] * (q[:, h // 2, :] @ S0[h].T) for h in range(Hv)], axis=1)
+    ref_s = np.exp(gam[-1])[:, None, None] * S0
+    harness.assert_close(res["out"], ref_o, res["final_state"], ref_s[None], "beta = 0 closed form")
+
+
+def test_prefill_onehot_keys_associative_recall():
+    """g = 0, beta = 1, distinct one-hot keys: the state stores v_j in column j exactly, a query
+    equal to an earlier key returns that value, a repeated key overwrites."""
+    from gdn_inputs import Tokens, f32_to_bf16_bits, bf16_bits_to_f32
+    T, Hv = 100, 2
+    rng = np.random.default_rng(59)
+    cols = np.concatenate([rng.permutation(128)[:90], rng.integers(0, 128, 10)])  # the last ten repeat keys
+    k = np.zeros((T, 1, 128), np.float32)
+    k[np.arange(T), 0, cols] = 1.0
+    ask = np.array([cols[rng.integers(0, t + 1)] for t in range(T)])             # a key seen so far
+    q = np.zeros((T, 1, 128), np.float32)
+    q[np.arange(T), 0, ask] = 1.0
+    v = rng.standard_normal((T, Hv, 128)).astype(np.float32)
+    tok = Tokens(q=f32_to_bf16_bits(q), k=f32_to_bf16_bits(k), v=f32_to_bf16_bits(v), g=np.zeros((T, Hv), np.float32),
+                 beta=np.ones((T, Hv), np.float32), Hqk=1, Hv=Hv, dk=128, dv=128)
+    res = harness.run_prefill(dict(tokens=tok, cu_seqlens=make_cu_seqlens([T]), initial_state=None))
+    vb = bf16_bits_to_f32(tok.v).astype(np.float64)
+    ref_o = np.stack([vb[max(s for s in range(t + 1) if cols[s] == ask[t])] for t in range(T)])  # latest write wins
+    ref_s = np.zeros((1, Hv, 128, 128))
+    for c in range(128):
+        writes = [s for s in range(T) if cols[s] == c]
+        if writes:
+            ref_s[0, :, :, c] = vb[writes[-1]]
+    # the chunked path rounds its intermediate operands to bf16, so "exactly" means within the tolerances
+    e = harness.assert_close(res["out"], ref_o, res["final_state"], ref_s, "one-hot recall")
+    assert e["out_rel_fro"] < 5e-3 and e["state_rel_fro"] < 2e-3
+    # the token-serial kernel keeps everything in fp32: there the recall is exact to bf16 rounding of the output
+    rec = harness.run_prefill(dict(tokens=tok, cu_seqlens=make_cu_seqlens([T]), initial_state=None), recurrent=True)
+    np.testing.assert_array_equal(rec["out"], ref_o)
+    np.testing.assert_allclose(rec["final_state"], ref_s, rtol=0, atol=1e-6)
