@@ -28,7 +28,8 @@
  * one-hot-key associative recall, the per-step identity for S k, the
  * orthogonal-key closed form through library matmuls, split/packing invariance,
  * linearity, V-row independence, brute-force matrix products on tiny inputs, the
- * paper's K x V form coded separately, and a chunked WY/UT reformulation.
+ * paper's K x V form coded separately, a chunked WY/UT reformulation, and the affine
+ * dependence on the entering state through the written-out transition product.
  */
 #include <math.h>
 #include <pthread.h>

@@ -324,3 +324,28 @@ def test_gated_oracle_closed_forms_and_agreement_with_the_ungated_form():
     op, sp = oracle.prefill_gated(tok.q, tok.k, tok.v, a, b, A_log, dt_bias, make_cu_seqlens([1] * 12), st)
     np.testing.assert_array_equal(od, op)
     np.testing.assert_array_equal(sd, sp)
+
+
+# ---- affine in the state (the identity behind sequence-parallel prefill): with M_t the product of the
+#      per-token transitions and H_t the zero-state response,  S_t = S_in M_t + H_t,  o_t = H_t q_t + S_in (M_t q_t).
+#      M_t q_t and M_T come from running the oracle itself on the identity (dk x dk "state", v = 0).
+def test_state_enters_affinely_through_the_transition_product():
+    T, dk, dv = 23, 8, 5
+    q, k, v, g, beta, S_in = rand_head(T, dk, dv, 41)
+    o_full, s_full = run_single(q, k, v, g, beta, S_in)
+    o_zero, s_zero = run_single(q, k, v, g, beta, None)                           # H_t q_t, H_T
+    o_id, s_id = run_single(q, k, np.zeros((T, dk)), g, beta, np.eye(dk))         # M_t q_t, M_T (a dk x dk run)
+    np.testing.assert_allclose(o_full, o_zero + o_id @ S_in.T, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(s_full[0], S_in @ s_id[0] + s_zero[0], rtol=1e-12, atol=1e-14)
+    # and the transition product itself, written out: M_T = prod_t alpha_t (I - beta_t k_t k_t^T)
+    M = np.eye(dk)
+    for t in range(T):
+        M = np.exp(g[t]) * (M @ (np.eye(dk) - beta[t] * np.outer(k[t], k[t])))
+    np.testing.assert_allclose(s_id[0], M, rtol=1e-12, atol=1e-14)
+    # two pieces joined: state after piece 1 enters piece 2
+    T1 = 9
+    _, s1 = run_single(q[:T1], k[:T1], v[:T1], g[:T1], beta[:T1], S_in)
+    o2_zero, s2_zero = run_single(q[T1:], k[T1:], v[T1:], g[T1:], beta[T1:], None)
+    o2_id, s2_id = run_single(q[T1:], k[T1:], np.zeros((T - T1, dk)), g[T1:], beta[T1:], np.eye(dk))
+    np.testing.assert_allclose(o_full[T1:], o2_zero + o2_id @ s1[0].T, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(s_full[0], s1[0] @ s2_id[0] + s2_zero[0], rtol=1e-12, atol=1e-14)
