@@ -15,7 +15,7 @@ constexpr int kStatusTimeout = 1;  // device status: a bounded wait ran out
 
 constexpr int kAssumedSMs = 148;   // co-resident chain CTAs the segment split is sized for
 constexpr int kMaxSegments = 8;    // segments a sequence is split into at most
-constexpr int kMinSegChunks = 4;   // a segment is at least this many chunks long
+constexpr int kMinSegChunks = 8;   // a segment is at least this many chunks long (shorter runs cost more in the scan than they save: measured)
 
 struct WsLayout {
     int nc_max;

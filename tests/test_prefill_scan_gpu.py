@@ -2,7 +2,7 @@
 chunk-run transitions) against the fp64 CPU oracle, through the C ABI.
 
 The library picks the number of runs from (sequences x value heads) and the longest sequence, so
-the shapes below are what selects 2, 4, 5 and 8 runs; GDN_PREFILL_MAX_SEGMENTS=1 switches the
+the shapes below are what selects 2, 3, 4, 5 and 8 runs; GDN_PREFILL_MAX_SEGMENTS=1 switches the
 split off for the A/B comparison."""
 import os
 
@@ -33,16 +33,16 @@ def check(cfg, what, **kw):
     return e, res
 
 
-# (lengths, Hqk, Hv): runs chosen = min((148 / (N Hv) + 1) / 2, 8, chunks / 4)
+# (lengths, Hqk, Hv): runs chosen = min((148 / (N Hv) + 1) / 2, 8, chunks of the longest sequence / 8)
 SHAPES = [
-    ([512], 4, 8, "8 chunks -> 2 runs"),
-    ([1024], 4, 8, "16 chunks -> 4 runs"),
-    ([2048], 4, 8, "32 chunks -> 8 runs"),
-    ([1000], 4, 8, "ragged tail, 16 chunks -> 4 runs of 4"),
-    ([1217], 2, 4, "20 chunks -> 5 runs, ragged"),
-    ([1100], 8, 16, "18 chunks, 16 heads -> 4 runs (5,5,5,3)"),
-    ([1500, 700], 4, 8, "two sequences -> 5 runs each; the short one has runs of 3, 3, 3, 2, 0 chunks"),
-    ([900, 0, 64], 2, 4, "an empty sequence and a one-chunk sequence beside a split one"),
+    ([1024], 4, 8, "16 chunks -> 2 runs"),
+    ([2048], 4, 8, "32 chunks -> 4 runs"),
+    ([4096], 4, 8, "64 chunks -> 8 runs"),
+    ([2000], 4, 8, "ragged tail, 32 chunks -> 4 runs of 8"),
+    ([2434], 2, 4, "39 chunks -> 4 runs (10, 10, 10, 9), ragged"),
+    ([2200], 8, 16, "35 chunks, 16 heads -> 4 runs (9, 9, 9, 8)"),
+    ([3000, 1400], 4, 8, "two sequences -> 5 runs each; the short one has runs of 5, 5, 5, 5, 2 chunks"),
+    ([1800, 0, 64], 2, 4, "an empty sequence and a one-chunk sequence beside one split into 3 runs"),
     ([1024], 8, 8, "one value head per key head"),
     ([1024], 2, 8, "four value heads per key head"),
     ([1024], 1, 3, "three value heads on one key head (an unpaired head in the intra-chunk kernel)"),
@@ -57,10 +57,10 @@ def test_split_prefill_matches_oracle(lengths, Hqk, Hv, what, gate_mean):
 
 
 def test_split_prefill_zero_initial_state_and_no_final_state():
-    cfg = custom([1024], 4, 8, seed=3, initial=False, gate_mean=5.0)
+    cfg = custom([2048], 4, 8, seed=3, initial=False, gate_mean=5.0)
     check(cfg, "zero initial state, 4 runs")
     check(cfg, "final state not requested, 4 runs", want_final=False)
-    cfg2 = custom([512], 4, 8, seed=4, gate_mean=5.0)
+    cfg2 = custom([1024], 4, 8, seed=4, gate_mean=5.0)
     check(cfg2, "final state not requested, 2 runs", want_final=False)
 
 
@@ -71,7 +71,7 @@ def test_split_prefill_full_size_long_sequence():
 
 def test_split_and_unsplit_agree():
     cfg = custom([2048], 4, 8, seed=21, gate_mean=6.0)
-    _, a = check(cfg, "8 runs")
+    _, a = check(cfg, "4 runs")
     os.environ["GDN_PREFILL_MAX_SEGMENTS"] = "1"
     try:
         _, b = check(cfg, "1 run")
@@ -85,7 +85,7 @@ def test_split_and_unsplit_agree():
 
 def test_split_prefill_correlated_keys():
     """Keys sharing a common direction: transitions far from a multiple of the identity."""
-    check(custom([1024], 4, 8, seed=23, gate_mean=6.0, key_correlation=0.5), "correlated keys, 4 runs")
+    check(custom([2048], 4, 8, seed=23, gate_mean=6.0, key_correlation=0.5), "correlated keys, 4 runs")
 
 
 def test_split_prefill_repeated_calls_reuse_workspace():
@@ -100,7 +100,7 @@ def test_split_prefill_repeated_calls_reuse_workspace():
 def test_split_prefill_strong_decay_underflows_cleanly(gate_mean):
     """g ~ -4 (-12) per token: cumulative decays underflow to zero inside a chunk, the transition of a
     run is exactly zero, and nothing may turn into NaN or Inf on the way."""
-    cfg = custom([1024], 4, 8, seed=37, gate_mean=gate_mean)
+    cfg = custom([2048], 4, 8, seed=37, gate_mean=gate_mean)
     _, res = check(cfg, "strong decay, 4 runs")
     assert np.isfinite(res["out"]).all() and np.isfinite(res["final_state"]).all()
 
