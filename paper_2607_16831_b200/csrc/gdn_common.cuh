@@ -62,14 +62,16 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// Function attributes (dynamic shared memory above 48 KB) are per device: returns true the first
-// time it is asked about `flags` on the current device, so the caller sets them then.
-inline bool first_use_on_device(bool (&flags)[64]) {
+// Function attributes (dynamic shared memory above 48 KB) are per device.  set_attrs_once runs `set`
+// the first time it is called with `flags` on the current device and remembers success only.
+template <typename F>
+inline cudaError_t set_attrs_once(bool (&flags)[64], F set) {
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;  // unknown: set them again
-    if (flags[dev]) return false;
-    flags[dev] = true;
-    return true;
+    const bool known = cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64;
+    if (known && flags[dev]) return cudaSuccess;
+    const cudaError_t e = set();
+    if (e == cudaSuccess && known) flags[dev] = true;
+    return e;
 }
 
 // GDN_NO_PDL=1 in the environment launches everything the ordinary way.

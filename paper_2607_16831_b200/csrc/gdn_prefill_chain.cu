@@ -590,11 +590,10 @@ cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, c
                                  const WsLayout& L, int num_seqs, int Hqk, int Hv, int segs, const ChainPartial& part,
                                  cudaStream_t st) {
     static bool attr_done[64];
-    if (first_use_on_device(attr_done)) {
-        cudaError_t e = cudaFuncSetAttribute(gdn_prefill_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kChainSmem);
-        if (e != cudaSuccess) return e;
-    }
+    if (cudaError_t e = set_attrs_once(attr_done, [] {
+            return cudaFuncSetAttribute(gdn_prefill_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kChainSmem);
+        }))
+        return e;
     const int per_seq = part.H ? 2 : 2 * segs - 1;
     gdn_prefill_chain_kernel<<<(unsigned)((long long)num_seqs * per_seq * Hv), kChainThreads, kChainSmem, st>>>(
         mq, mk, mv, initial_state, (uint16_t*)out, final_state, ws, L, Hqk, Hv, segs, part);

@@ -531,11 +531,10 @@ cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, c
                                  int Hv, const int32_t* cu_if_no_table, int num_seqs, int total_tokens,
                                  cudaStream_t st) {
     static bool attr_done[64];
-    if (first_use_on_device(attr_done)) {
-        cudaError_t e = cudaFuncSetAttribute(gdn_prefill_intra_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kIntraSmem);
-        if (e != cudaSuccess) return e;
-    }
+    if (cudaError_t e = set_attrs_once(attr_done, [] {
+            return cudaFuncSetAttribute(gdn_prefill_intra_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kIntraSmem);
+        }))
+        return e;
     const int G = Hv / Hqk;
     dim3 grid(L.nc_max, Hqk * ((G + 1) / 2));
     gdn_prefill_intra_kernel<<<grid, kIntraThreads, kIntraSmem, st>>>(mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv,

@@ -288,13 +288,12 @@ gdn_prefill_fixup_kernel(const __grid_constant__ CUtensorMap map_out, const __gr
 
 static cudaError_t scan_attrs() {
     static bool attr_done[64];
-    if (first_use_on_device(attr_done)) {
+    return set_attrs_once(attr_done, [] {
         cudaError_t e = cudaFuncSetAttribute(gdn_prefill_fixup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFixSmem);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(gdn_prefill_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, combine_smem(2));
-        if (e != cudaSuccess) return e;
-    }
-    return cudaSuccess;
+        return e;
+    });
 }
 
 cudaError_t launch_prefill_scan(const CUtensorMap& mout, const CUtensorMap& mqt, void* out, float* final_state,
