@@ -48,6 +48,11 @@ def _load():
         lib.gdn_oracle_prefill_gated.restype = I
         lib.gdn_oracle_decode_gated.argtypes = [P] * 10 + [I] * 6
         lib.gdn_oracle_decode_gated.restype = I
+        D = ctypes.c_double
+        lib.gdn_oracle_prefill_fused.argtypes = [P] * 11 + [I] * 5 + [D, I, I]
+        lib.gdn_oracle_prefill_fused.restype = I
+        lib.gdn_oracle_decode_fused.argtypes = [P] * 10 + [I] * 5 + [D, I, I]
+        lib.gdn_oracle_decode_fused.restype = I
         _lib = lib
     return _lib
 
@@ -150,4 +155,49 @@ def decode_gated(q, k, v, a, b, A_log, dt_bias, state_in, threads: Optional[int]
                                          threads or default_threads())
     if rc != 0:
         raise ValueError("gdn_oracle_decode_gated: bad arguments")
+    return out, so
+
+
+def prefill_fused(q, k, v, a, b, A_log, dt_bias, cu_seqlens, initial_state=None, scale=1.0, qk_l2norm=False,
+                  want_final=True, threads: Optional[int] = None):
+    """As `prefill_gated` with the fused front end: with qk_l2norm, q and k of every (token, head)
+    are divided by sqrt(sum of squares + 1e-6); q is then multiplied by `scale` (all in fp64).
+    A_log = dt_bias = None: a and b are the log-decay g and beta themselves."""
+    q, k, v = _c(q, np.uint16), _c(k, np.uint16), _c(v, np.uint16)
+    a, b = _c(a, np.float32), _c(b, np.float32)
+    if A_log is not None:
+        A_log, dt_bias = _c(A_log, np.float32), _c(dt_bias, np.float32)
+    cu = _c(cu_seqlens, np.int32)
+    T, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    N = cu.shape[0] - 1
+    assert a.shape == (T, Hv) and b.shape == (T, Hv)
+    if initial_state is not None:
+        initial_state = _c(initial_state, np.float32)
+    out = np.zeros((T, Hv, dv), dtype=np.float64)
+    fin = np.zeros((N, Hv, dv, dk), dtype=np.float64) if want_final else None
+    rc = _load().gdn_oracle_prefill_fused(_ptr(q), _ptr(k), _ptr(v), _ptr(a), _ptr(b), _ptr(A_log), _ptr(dt_bias),
+                                          _ptr(cu), _ptr(initial_state), _ptr(out), _ptr(fin), N, Hqk, Hv, dk, dv,
+                                          float(scale), int(bool(qk_l2norm)), threads or default_threads())
+    if rc != 0:
+        raise ValueError("gdn_oracle_prefill_fused: bad arguments")
+    return out, fin
+
+
+def decode_fused(q, k, v, a, b, A_log, dt_bias, state_in, scale=1.0, qk_l2norm=False,
+                 threads: Optional[int] = None):
+    q, k, v = _c(q, np.uint16), _c(k, np.uint16), _c(v, np.uint16)
+    a, b = _c(a, np.float32), _c(b, np.float32)
+    if A_log is not None:
+        A_log, dt_bias = _c(A_log, np.float32), _c(dt_bias, np.float32)
+    state_in = _c(state_in, np.float32)
+    B, Hqk, dk = q.shape
+    _, Hv, dv = v.shape
+    out = np.zeros((B, Hv, dv), dtype=np.float64)
+    so = np.zeros((B, Hv, dv, dk), dtype=np.float64)
+    rc = _load().gdn_oracle_decode_fused(_ptr(q), _ptr(k), _ptr(v), _ptr(a), _ptr(b), _ptr(A_log), _ptr(dt_bias),
+                                         _ptr(state_in), _ptr(so), _ptr(out), B, Hqk, Hv, dk, dv, float(scale),
+                                         int(bool(qk_l2norm)), threads or default_threads())
+    if rc != 0:
+        raise ValueError("gdn_oracle_decode_fused: bad arguments")
     return out, so

@@ -24,12 +24,20 @@
  * The *_gated entry points take the paper's raw gate inputs (Section 3.2, first two lines:
  * g = exp(-exp(A_log) softplus(a + b_dt)), beta = sigmoid(b)) and evaluate them in fp64.
  *
+ * The *_fused entry points add the operator's front end as deployed in a layer, which the paper does
+ * not spell out (it is this library's stated interface convention, not a formula of the paper):
+ * with qk_l2norm, q and k of every (token, head) are divided by sqrt(sum of squares + 1e-6); q is
+ * then multiplied by `scale`.  Both happen in fp64 on the widened bf16 values, before the five lines
+ * above.  A_log = dt_bias = NULL there means that g and beta are given directly.
+ *
  * Pins (tests/test_oracle_pins.py): one-token closed form, beta = 0 pure decay,
  * one-hot-key associative recall, the per-step identity for S k, the
  * orthogonal-key closed form through library matmuls, split/packing invariance,
  * linearity, V-row independence, brute-force matrix products on tiny inputs, the
  * paper's K x V form coded separately, a chunked WY/UT reformulation, and the affine
- * dependence on the entering state through the written-out transition product.
+ * dependence on the entering state through the written-out transition product; for the fused
+ * front end: linearity in scale, agreement with the separately coded forms run on inputs
+ * normalised with library routines, invariance to rescaling q and k, recall with non-unit one-hot keys.
  */
 #include <math.h>
 #include <pthread.h>
@@ -48,6 +56,9 @@ typedef struct {
     const uint16_t *q, *k, *v;
     const float *g, *beta;          /* log-decay and write strength, or (gated entry points) the raw a and b */
     const float *A_log, *dt_bias;   /* per value head; NULL unless the raw-gate form is used */
+    int fused;                      /* fused front end: normalisation and scale below apply */
+    int qk_l2norm;
+    double scale;
     const int32_t *cu_seqlens; /* NULL => decode: sequence n is the single token n */
     const float *initial_state;
     double *out, *final_state;
@@ -75,6 +86,21 @@ static void run_unit(const job_t *J, int n, int h, double *S, double *kk, double
         for (int c = 0; c < dk; ++c) {
             kk[c] = bf16_to_double(kt[c]);
             qq[c] = bf16_to_double(qt[c]);
+        }
+        if (J->fused) {
+            if (J->qk_l2norm) { /* x <- x / sqrt(sum x^2 + 1e-6), for k and for q */
+                double sk = 0.0, sq = 0.0;
+                for (int c = 0; c < dk; ++c) {
+                    sk += kk[c] * kk[c];
+                    sq += qq[c] * qq[c];
+                }
+                const double nk = sqrt(sk + 1e-6), nq = sqrt(sq + 1e-6);
+                for (int c = 0; c < dk; ++c) {
+                    kk[c] /= nk;
+                    qq[c] /= nq;
+                }
+            }
+            for (int c = 0; c < dk; ++c) qq[c] *= J->scale;
         }
         double alpha, beta;
         if (J->A_log) {
@@ -203,5 +229,40 @@ int gdn_oracle_decode_gated(const uint16_t *q, const uint16_t *k, const uint16_t
     J.out = out; J.final_state = state_out;
     J.num_seqs = B; J.Hqk = Hqk; J.Hv = Hv; J.dk = dk; J.dv = dv;
     if (!state_in || !A_log || !dt_bias) return 1;
+    return run_job(&J, num_threads);
+}
+
+/* Fused front end: raw gates when A_log and dt_bias are given (both or neither), q/k L2
+ * normalisation when qk_l2norm != 0, q multiplied by scale.  Otherwise as the entry points above. */
+int gdn_oracle_prefill_fused(const uint16_t *q, const uint16_t *k, const uint16_t *v, const float *a,
+                             const float *b, const float *A_log, const float *dt_bias,
+                             const int32_t *cu_seqlens, const float *initial_state, double *out,
+                             double *final_state, int num_seqs, int Hqk, int Hv, int dk, int dv,
+                             double scale, int qk_l2norm, int num_threads) {
+    job_t J;
+    memset(&J, 0, sizeof J);
+    J.q = q; J.k = k; J.v = v; J.g = a; J.beta = b; J.A_log = A_log; J.dt_bias = dt_bias;
+    J.fused = 1; J.scale = scale; J.qk_l2norm = qk_l2norm;
+    J.cu_seqlens = cu_seqlens;
+    J.initial_state = initial_state;
+    J.out = out; J.final_state = final_state;
+    J.num_seqs = num_seqs; J.Hqk = Hqk; J.Hv = Hv; J.dk = dk; J.dv = dv;
+    if (!cu_seqlens || (A_log == NULL) != (dt_bias == NULL)) return 1;
+    return run_job(&J, num_threads);
+}
+
+int gdn_oracle_decode_fused(const uint16_t *q, const uint16_t *k, const uint16_t *v, const float *a,
+                            const float *b, const float *A_log, const float *dt_bias,
+                            const float *state_in, double *state_out, double *out, int B, int Hqk,
+                            int Hv, int dk, int dv, double scale, int qk_l2norm, int num_threads) {
+    job_t J;
+    memset(&J, 0, sizeof J);
+    J.q = q; J.k = k; J.v = v; J.g = a; J.beta = b; J.A_log = A_log; J.dt_bias = dt_bias;
+    J.fused = 1; J.scale = scale; J.qk_l2norm = qk_l2norm;
+    J.cu_seqlens = NULL;
+    J.initial_state = state_in;
+    J.out = out; J.final_state = state_out;
+    J.num_seqs = B; J.Hqk = Hqk; J.Hv = Hv; J.dk = dk; J.dv = dv;
+    if (!state_in || (A_log == NULL) != (dt_bias == NULL)) return 1;
     return run_job(&J, num_threads);
 }

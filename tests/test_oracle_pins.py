@@ -349,3 +349,84 @@ def test_state_enters_affinely_through_the_transition_product():
     o2_id, s2_id = run_single(q[T1:], k[T1:], np.zeros((T - T1, dk)), g[T1:], beta[T1:], np.eye(dk))
     np.testing.assert_allclose(o_full[T1:], o2_zero + o2_id @ s1[0].T, rtol=1e-12, atol=1e-14)
     np.testing.assert_allclose(s_full[0], s1[0] @ s2_id[0] + s2_zero[0], rtol=1e-12, atol=1e-14)
+
+
+# ---- fused front end: q/k L2 normalisation (x / sqrt(sum x^2 + 1e-6)) and a scale on q
+def test_fused_front_end_scale_normalisation_and_recall():
+    tok = make_tokens(40, 2, 4, dk=16, dv=6, seed=200)
+    # make the norms far from 1 and different per token, exactly in bf16 (powers of two per token)
+    rng = np.random.default_rng(200)
+    pw_k = (2.0 ** rng.integers(-2, 4, size=(40, 2, 1))).astype(np.float32)
+    pw_q = (2.0 ** rng.integers(-3, 3, size=(40, 2, 1))).astype(np.float32)
+    kb = f32_to_bf16_bits(bf16_bits_to_f32(tok.k) * pw_k)
+    qb = f32_to_bf16_bits(bf16_bits_to_f32(tok.q) * pw_q)
+    init = make_state(2, 4, 16, 6, seed=200, sd=0.3)
+    cu = make_cu_seqlens([29, 11])
+    # (1) switched off it is the plain definition, bit for bit
+    o0, s0 = oracle.prefill(qb, kb, tok.v, tok.g, tok.beta, cu, init)
+    o1, s1 = oracle.prefill_fused(qb, kb, tok.v, tok.g, tok.beta, None, None, cu, init, scale=1.0, qk_l2norm=False)
+    np.testing.assert_array_equal(o0, o1)
+    np.testing.assert_array_equal(s0, s1)
+    # (2) scale multiplies the outputs and leaves the states alone (o = S q is linear in q; S does not see q)
+    o2, s2 = oracle.prefill_fused(qb, kb, tok.v, tok.g, tok.beta, None, None, cu, init, scale=0.375, qk_l2norm=False)
+    np.testing.assert_allclose(o2, 0.375 * o0, rtol=1e-13, atol=1e-300)
+    np.testing.assert_array_equal(s2, s0)
+    # (3) normalisation: the separately coded forms, fed inputs normalised here with library routines
+    o3, s3 = oracle.prefill_fused(qb, kb, tok.v, tok.g, tok.beta, None, None, cu, init, scale=0.25, qk_l2norm=True)
+    q64 = bf16_bits_to_f32(qb).astype(np.float64)
+    k64 = bf16_bits_to_f32(kb).astype(np.float64)
+    qn = 0.25 * q64 / np.sqrt(np.einsum("thd,thd->th", q64, q64) + 1e-6)[..., None]
+    kn = k64 / np.sqrt(np.einsum("thd,thd->th", k64, k64) + 1e-6)[..., None]
+    for n, (t0, t1) in enumerate([(0, 29), (29, 40)]):
+        for h in range(4):
+            v64 = bf16_bits_to_f32(tok.v[t0:t1, h]).astype(np.float64)
+            g64, b64 = tok.g[t0:t1, h].astype(np.float64), tok.beta[t0:t1, h].astype(np.float64)
+            S0 = init[n, h].astype(np.float64)
+            for form in (R.paper_form, lambda *a: R.chunked(*a, C=8)):
+                ro, rs = form(qn[t0:t1, h // 2], kn[t0:t1, h // 2], v64, g64, b64, S0)
+                np.testing.assert_allclose(o3[t0:t1, h], ro, rtol=1e-10, atol=1e-13)
+                np.testing.assert_allclose(s3[n, h], rs, rtol=1e-10, atol=1e-13)
+    # the norms really were far from 1: without normalisation the result differs grossly
+    assert rel_fro(0.25 * o0, o3) > 0.1
+    # (4) invariance: rescaling q and k per token by powers of two changes nothing but the 1e-6 term
+    o4, s4 = oracle.prefill_fused(tok.q, tok.k, tok.v, tok.g, tok.beta, None, None, cu, init, scale=0.25, qk_l2norm=True)
+    # tok.k has norm 1 and tok.q norm 1/4: the 1e-6 under the root moves the unit vectors by < 1e-5 relative
+    assert rel_fro(o3, o4) < 2e-4 and rel_fro(s3, s4) < 2e-4
+    big_k = f32_to_bf16_bits(bf16_bits_to_f32(tok.k) * np.float32(1024.0))
+    big_q = f32_to_bf16_bits(bf16_bits_to_f32(tok.q) * np.float32(4096.0))
+    big_k2 = f32_to_bf16_bits(bf16_bits_to_f32(big_k) * pw_k)
+    big_q2 = f32_to_bf16_bits(bf16_bits_to_f32(big_q) * pw_q)
+    o5, s5 = oracle.prefill_fused(big_q, big_k, tok.v, tok.g, tok.beta, None, None, cu, init, scale=0.25, qk_l2norm=True)
+    o6, s6 = oracle.prefill_fused(big_q2, big_k2, tok.v, tok.g, tok.beta, None, None, cu, init, scale=0.25, qk_l2norm=True)
+    assert rel_fro(o6, o5) < 1e-10 and rel_fro(s6, s5) < 1e-10   # 1e-6 against squared norms >= 6e4
+    # (5) recall with one-hot keys of magnitude 3: normalised they are unit vectors, so with g = 0, beta = 1
+    #     the state returns v_s for q = k_s exactly (up to the 1e-6 under the root: 1 - 9/(9+1e-6) ~ 1e-7)
+    T, dk, dv = 6, 8, 5
+    idx = np.array([2, 5, 0, 7, 3, 5])                      # key 5 is written twice: the second write wins
+    kk = np.zeros((T, 1, dk), np.float32)
+    kk[np.arange(T), 0, idx] = 3.0
+    vv = rng.standard_normal((T, 1, dv)).astype(np.float32)
+    vb, v_exact = round_bf16(vv)
+    oo, ss = oracle.prefill_fused(f32_to_bf16_bits(kk), f32_to_bf16_bits(kk), vb, np.zeros((T, 1), np.float32),
+                                  np.ones((T, 1), np.float32), None, None, make_cu_seqlens([T]), None,
+                                  scale=2.0, qk_l2norm=True)
+    np.testing.assert_allclose(oo[:, 0], 2.0 * v_exact[:, 0], rtol=1e-6, atol=1e-12)   # o_t = scale * v_t
+    last = {int(j): t for t, j in enumerate(idx)}
+    for j, t in last.items():
+        np.testing.assert_allclose(ss[0, 0][:, j], v_exact[t, 0], rtol=1e-6, atol=1e-12)
+    # (6) raw gates and the front end together; decode form = one-token sequences
+    from gdn_inputs import make_raw_gates
+    a, b, A_log, dt_bias = make_raw_gates(40, 4, seed=200)
+    o7, s7 = oracle.prefill_fused(qb, kb, tok.v, a, b, A_log, dt_bias, cu, init, scale=0.25, qk_l2norm=True)
+    o8, s8 = oracle.prefill_fused(qb, kb, tok.v, a, b, A_log, dt_bias, cu, init, scale=1.0, qk_l2norm=True)
+    np.testing.assert_allclose(o7, 0.25 * o8, rtol=1e-13, atol=1e-300)
+    x = a.astype(np.float64) + dt_bias.astype(np.float64)[None, :]
+    g64 = (-np.exp(A_log.astype(np.float64))[None, :] * np.logaddexp(0.0, x)).astype(np.float32)
+    beta64 = (1.0 / (1.0 + np.exp(-b.astype(np.float64)))).astype(np.float32)
+    o9, s9 = oracle.prefill_fused(qb, kb, tok.v, g64, beta64, None, None, cu, init, scale=0.25, qk_l2norm=True)
+    assert rel_fro(o7, o9) < 1e-6 and rel_fro(s7, s9) < 1e-6
+    st = make_state(40, 4, 16, 6, seed=201, sd=0.3)
+    od, sd = oracle.decode_fused(qb, kb, tok.v, a, b, A_log, dt_bias, st, scale=0.25, qk_l2norm=True)
+    op, sp = oracle.prefill_fused(qb, kb, tok.v, a, b, A_log, dt_bias, make_cu_seqlens([1] * 40), st, scale=0.25, qk_l2norm=True)
+    np.testing.assert_array_equal(od, op)
+    np.testing.assert_array_equal(sd, sp)
