@@ -181,7 +181,7 @@ def decode_buffers(B, seed=0, min_footprint=600e6):
     return cfg, d, s_in, s_out, out, nbuf
 
 
-def bench_prefill(name, peaks, reps, env=None, lengths=None, **over):
+def bench_prefill(name, peaks, reps, env=None, lengths=None, fused=False, **over):
     """Whole-call device time of gdn_prefill (chunk table + intra-chunk + chain kernels, plus the
     scan over runs of chunks when the library splits long sequences).  `env` holds library
     switches set for the duration of this measurement; `lengths` replaces the workload's
@@ -214,6 +214,14 @@ def bench_prefill(name, peaks, reps, env=None, lengths=None, **over):
 
     def call():
         gdn.gdn_prefill(d["q"], d["k"], d["v"], d["g"], d["beta"], cu, init, out, fin, max_len, ws)
+
+    if fused:  # raw gates, q/k L2 normalisation and a scale on q inside the kernels
+        from gdn_inputs import make_raw_gates
+        ra, rb, rA, rdt = (torch.from_numpy(x).cuda() for x in make_raw_gates(tok.T, tok.Hv))
+
+        def call():
+            gdn.gdn_prefill_fused(d["q"], d["k"], d["v"], ra, rb, rA, rdt, cu, init, out, fin, max_len, ws,
+                                  scale=0.5, qk_l2norm=True)
 
     for _ in range(3):
         call()
@@ -415,6 +423,10 @@ def run_gpu(args):
                                                             sog[i % nbg], oog), iters=40)
         line["decode_gated_b64"] = {"us_per_call": med, "state_gbs": 64 * STATE_BYTES_PER_ITEM / med / 1e3,
                                     "note": "gdn_decode_gated: g and beta computed in the kernel from raw gate inputs"}
+        med, mn = time_graph(lambda i: gdn.gdn_decode_fused(dg["q"], dg["k"], dg["v"], ra, rb, rA, rdt, sig[i % nbg],
+                                                            sog[i % nbg], oog, scale=0.5, qk_l2norm=True), iters=40)
+        line["decode_fused_b64"] = {"us_per_call": med, "state_gbs": 64 * STATE_BYTES_PER_ITEM / med / 1e3,
+                                    "note": "gdn_decode_fused: raw gates, q/k L2 normalisation and the scale on q in the kernel"}
         del cfg_g, dg, sig, sog, oog
         torch.cuda.empty_cache()
         # ---- multi-token decode: T = 4 tokens per item in one pass over the state
@@ -443,6 +455,10 @@ def run_gpu(args):
         pre.append(dict(bench_prefill("prefill_long", peaks, reps), variant="zero initial state"))
         pre.append(dict(bench_prefill("prefill_long", peaks, reps, initial=True), variant="N(0,0.02) initial state"))
         pre.append(dict(bench_prefill("prefill_varlen", peaks, reps), variant="16 sequences U[1,2048]"))
+        pre.append(dict(bench_prefill("prefill_long", peaks, reps, initial=True, fused=True),
+                        variant="gdn_prefill_fused (raw gates, q/k L2 norm, scale), N(0,0.02) initial state"))
+        pre.append(dict(bench_prefill("prefill_varlen", peaks, reps, fused=True),
+                        variant="gdn_prefill_fused, 16 sequences U[1,2048]"))
         pre.append(dict(bench_prefill("prefill_long", peaks, reps, env={"GDN_PREFILL_MAX_SEGMENTS": "1"}),
                         variant="zero initial state, sequence split switched off (one chain CTA per head)"))
         # smaller head counts (4 key / 8 value heads), where one sequence leaves even more of the GPU idle

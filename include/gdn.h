@@ -172,6 +172,29 @@ int gdn_prefill_gated(const void* q, const void* k, const void* v, const float* 
                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Both entry points with the whole front end of the operator fused in: the raw gates of Section
+ * 3.2 as in gdn_decode_gated / gdn_prefill_gated (pass A_log = dt_bias = NULL to give the log-decay g
+ * and beta themselves in a and b), and what a layer applies to q and k before the recurrence, which
+ * the paper leaves to the caller and this library defines as follows:
+ *   qk_l2norm != 0:  q and k of every (token, q/k head) are divided by sqrt(sum of squares + 1e-6),
+ *                    the sum over the 128 elements in fp32;
+ *   then q is multiplied by `scale` (finite; 1 = none).
+ * The kernels do not form normalised copies of q and k: the two per-token factors enter the dot
+ * products, the decay coefficients and the output scaling in fp32, so the result is that of the
+ * recurrence run on unrounded normalised inputs.  A zero vector stays zero.
+ * Errors as for the gated entry points; GDN_ERR_NULL also when exactly one of A_log, dt_bias is NULL;
+ * GDN_ERR_SHAPE when scale is not finite.
+ */
+int gdn_decode_fused(const void* q, const void* k, const void* v, const float* a, const float* b,
+                     const float* A_log, const float* dt_bias, const float* state_in, float* state_out, void* out,
+                     int B, int Hqk, int Hv, int dk, int dv, float scale, int qk_l2norm, void* stream);
+int gdn_prefill_fused(const void* q, const void* k, const void* v, const float* a, const float* b,
+                      const float* A_log, const float* dt_bias, const int32_t* cu_seqlens,
+                      const float* initial_state, void* out, float* final_state,
+                      int total_tokens, int num_seqs, int max_seqlen, int Hqk, int Hv, int dk, int dv,
+                      float scale, int qk_l2norm, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Token-serial prefill: the same inputs and outputs as gdn_prefill (no workspace),
  * computed by the per-token recurrence of Section 3.2 with the state rows held in
  * registers and split along V across thread blocks (the paper's own prefill shape).

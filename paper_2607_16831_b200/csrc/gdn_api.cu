@@ -8,14 +8,15 @@
 namespace gdn {
 cudaError_t decode_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
                             const float* A_log, const float* dt_bias, const float* s_in, float* s_out, void* out,
-                            int B, int Hqk, int Hv, int variant, cudaStream_t st);
+                            int B, int Hqk, int Hv, int variant, QkFront fr, cudaStream_t st);
 cudaError_t decode_multi_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
                                   const float* s_in, float* s_out, void* out, int B, int T, int Hqk, int Hv,
                                   cudaStream_t st);
 cudaError_t prefill_recurrent_dispatch(const void* q, const void* k, const void* v, const float* g,
-                                       const float* beta, const int32_t* cu_seqlens, const float* initial_state,
-                                       void* out, float* final_state, int total_tokens, int num_seqs, int Hqk,
-                                       int Hv, int* status_word, cudaStream_t st);
+                                       const float* beta, const float* A_log, const float* dt_bias,
+                                       const int32_t* cu_seqlens, const float* initial_state, void* out,
+                                       float* final_state, int total_tokens, int num_seqs, int Hqk, int Hv,
+                                       int* status_word, QkFront fr, cudaStream_t st);
 size_t prefill_chunked_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv, bool allow_split);
 cudaError_t prefill_partial_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
                                      const int32_t* cu_seqlens, void* out0, void* qt, float* H, float* P,
@@ -31,7 +32,7 @@ cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v
                                      const int32_t* cu_seqlens, const float* initial_state,
                                      void* out, float* final_state, int total_tokens, int num_seqs,
                                      int max_seqlen, int Hqk, int Hv, void* workspace, size_t workspace_bytes,
-                                     bool allow_split, cudaStream_t st);
+                                     bool allow_split, QkFront fr, cudaStream_t st);
 
 // 1 = sm_100 family, 0 = other, -1 = unknown yet.  Indexed by device ordinal.
 static int g_device_ok[64] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1,
@@ -68,7 +69,7 @@ static int check_heads(int Hqk, int Hv, int dk, int dv) {
 
 static int decode_impl(const void* q, const void* k, const void* v, const float* g, const float* beta,
                        const float* A_log, const float* dt_bias, bool gated, const float* state_in, float* state_out,
-                       void* out, int B, int Hqk, int Hv, int dk, int dv, int variant, void* stream) {
+                       void* out, int B, int Hqk, int Hv, int dk, int dv, int variant, QkFront fr, void* stream) {
     if (B < 0) return GDN_ERR_SHAPE;
     if (int rc = check_heads(Hqk, Hv, dk, dv)) return rc;
     if (B == 0) return GDN_OK;
@@ -81,7 +82,7 @@ static int decode_impl(const void* q, const void* k, const void* v, const float*
     if ((long long)B * Hv * 32 > 0x7fffffffLL) return GDN_ERR_SHAPE;
     if (!device_supported()) return GDN_ERR_UNSUPPORTED;
     return cuda_status(decode_dispatch(q, k, v, g, beta, gated ? A_log : nullptr, gated ? dt_bias : nullptr, state_in,
-                                       state_out, out, B, Hqk, Hv, variant, (cudaStream_t)stream), "gdn_decode");
+                                       state_out, out, B, Hqk, Hv, variant, fr, (cudaStream_t)stream), "gdn_decode");
 }
 
 static int check_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
@@ -147,7 +148,7 @@ int gdn_decode(const void* q, const void* k, const void* v, const float* g, cons
                const float* state_in, float* state_out, void* out, int B, int Hqk, int Hv, int dk, int dv,
                void* stream) {
     return decode_impl(q, k, v, g, beta, nullptr, nullptr, false, state_in, state_out, out, B, Hqk, Hv, dk, dv, -1,
-                       stream);
+                       QkFront{1.f, 0}, stream);
 }
 
 int gdn_decode_variant(const void* q, const void* k, const void* v, const float* g, const float* beta,
@@ -155,7 +156,7 @@ int gdn_decode_variant(const void* q, const void* k, const void* v, const float*
                        int variant, void* stream) {
     if (variant < 0 || variant >= gdn_decode_num_variants()) return GDN_ERR_SHAPE;
     return decode_impl(q, k, v, g, beta, nullptr, nullptr, false, state_in, state_out, out, B, Hqk, Hv, dk, dv, variant,
-                       stream);
+                       QkFront{1.f, 0}, stream);
 }
 
 int gdn_decode_num_variants(void) { return 12; }
@@ -196,20 +197,65 @@ int gdn_prefill(const void* q, const void* k, const void* v, const float* g, con
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
         return GDN_ERR_WORKSPACE;
     if (prefer_token_serial(num_seqs, Hv, max_seqlen)) {
-        return cuda_status(prefill_recurrent_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
-                                                      total_tokens, num_seqs, Hqk, Hv, static_cast<int*>(workspace),
+        return cuda_status(prefill_recurrent_dispatch(q, k, v, g, beta, nullptr, nullptr, cu_seqlens, initial_state,
+                                                      out, final_state, total_tokens, num_seqs, Hqk, Hv,
+                                                      static_cast<int*>(workspace), QkFront{1.f, 0},
                                                       (cudaStream_t)stream),
                            "gdn_prefill (token-serial)");
     }
     return cuda_status(prefill_chunked_dispatch(q, k, v, g, beta, nullptr, nullptr, cu_seqlens, initial_state, out,
                                                 final_state, total_tokens, num_seqs, max_seqlen, Hqk, Hv, workspace,
-                                                workspace_bytes, true, (cudaStream_t)stream), "gdn_prefill");
+                                                workspace_bytes, true, QkFront{1.f, 0}, (cudaStream_t)stream),
+                       "gdn_prefill");
 }
 
 int gdn_decode_gated(const void* q, const void* k, const void* v, const float* a, const float* b, const float* A_log,
                      const float* dt_bias, const float* state_in, float* state_out, void* out, int B, int Hqk,
                      int Hv, int dk, int dv, void* stream) {
-    return decode_impl(q, k, v, a, b, A_log, dt_bias, true, state_in, state_out, out, B, Hqk, Hv, dk, dv, -1, stream);
+    return decode_impl(q, k, v, a, b, A_log, dt_bias, true, state_in, state_out, out, B, Hqk, Hv, dk, dv, -1,
+                       QkFront{1.f, 0}, stream);
+}
+
+// scale must be finite; qk_l2norm is a flag
+static bool front_ok(float scale) { return scale == scale && scale - scale == 0.f; }
+
+int gdn_decode_fused(const void* q, const void* k, const void* v, const float* a, const float* b, const float* A_log,
+                     const float* dt_bias, const float* state_in, float* state_out, void* out, int B, int Hqk,
+                     int Hv, int dk, int dv, float scale, int qk_l2norm, void* stream) {
+    if (!front_ok(scale)) return GDN_ERR_SHAPE;
+    if (B > 0 && ((A_log == nullptr) != (dt_bias == nullptr))) return GDN_ERR_NULL;
+    return decode_impl(q, k, v, a, b, A_log, dt_bias, A_log != nullptr, state_in, state_out, out, B, Hqk, Hv, dk, dv,
+                       -1, QkFront{scale, qk_l2norm != 0}, stream);
+}
+
+// gdn_prefill_gated and gdn_prefill_fused: raw gates when A_log / dt_bias are given, and the q/k front end
+static int prefill_front_impl(const void* q, const void* k, const void* v, const float* a, const float* b,
+                              const float* A_log, const float* dt_bias, bool gates_required,
+                              const int32_t* cu_seqlens, const float* initial_state, void* out, float* final_state,
+                              int total_tokens, int num_seqs, int max_seqlen, int Hqk, int Hv, int dk, int dv,
+                              QkFront fr, void* workspace, size_t workspace_bytes, void* stream, const char* name) {
+    // a missing gate parameter is reported ahead of the device check, like the other host-side errors
+    const bool gates_missing = gates_required ? (!A_log || !dt_bias) : ((A_log == nullptr) != (dt_bias == nullptr));
+    if (gates_missing && total_tokens >= 0 && num_seqs > 0 && max_seqlen >= 0 && check_heads(Hqk, Hv, dk, dv) == GDN_OK)
+        return GDN_ERR_NULL;
+    bool nothing = false;
+    if (int rc = check_prefill(q, k, v, a, b, cu_seqlens, initial_state, out, final_state, total_tokens, num_seqs,
+                               max_seqlen, Hqk, Hv, dk, dv, &nothing))
+        return rc;
+    if (nothing) return GDN_OK;
+    if ((reinterpret_cast<uintptr_t>(A_log) & 3u) || (reinterpret_cast<uintptr_t>(dt_bias) & 3u)) return GDN_ERR_ALIGN;
+    const size_t need = prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv, true);
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
+        return GDN_ERR_WORKSPACE;
+    if (prefer_token_serial(num_seqs, Hv, max_seqlen)) {
+        return cuda_status(prefill_recurrent_dispatch(q, k, v, a, b, A_log, dt_bias, cu_seqlens, initial_state, out,
+                                                      final_state, total_tokens, num_seqs, Hqk, Hv,
+                                                      static_cast<int*>(workspace), fr, (cudaStream_t)stream),
+                           name);
+    }
+    return cuda_status(prefill_chunked_dispatch(q, k, v, a, b, A_log, dt_bias, cu_seqlens, initial_state, out,
+                                                final_state, total_tokens, num_seqs, max_seqlen, Hqk, Hv, workspace,
+                                                workspace_bytes, true, fr, (cudaStream_t)stream), name);
 }
 
 int gdn_prefill_gated(const void* q, const void* k, const void* v, const float* a, const float* b,
@@ -217,19 +263,20 @@ int gdn_prefill_gated(const void* q, const void* k, const void* v, const float* 
                       const float* initial_state, void* out, float* final_state, int total_tokens, int num_seqs,
                       int max_seqlen, int Hqk, int Hv, int dk, int dv, void* workspace, size_t workspace_bytes,
                       void* stream) {
-    bool nothing = false;
-    if (int rc = check_prefill(q, k, v, a, b, cu_seqlens, initial_state, out, final_state, total_tokens, num_seqs,
-                               max_seqlen, Hqk, Hv, dk, dv, &nothing))
-        return rc;
-    if (nothing) return GDN_OK;
-    if (!A_log || !dt_bias) return GDN_ERR_NULL;
-    if ((reinterpret_cast<uintptr_t>(A_log) & 3u) || (reinterpret_cast<uintptr_t>(dt_bias) & 3u)) return GDN_ERR_ALIGN;
-    const size_t need = prefill_chunked_workspace_bytes(total_tokens, num_seqs, Hqk, Hv, true);
-    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u))
-        return GDN_ERR_WORKSPACE;
-    return cuda_status(prefill_chunked_dispatch(q, k, v, a, b, A_log, dt_bias, cu_seqlens, initial_state, out,
-                                                final_state, total_tokens, num_seqs, max_seqlen, Hqk, Hv, workspace,
-                                                workspace_bytes, true, (cudaStream_t)stream), "gdn_prefill_gated");
+    return prefill_front_impl(q, k, v, a, b, A_log, dt_bias, true, cu_seqlens, initial_state, out, final_state,
+                              total_tokens, num_seqs, max_seqlen, Hqk, Hv, dk, dv, QkFront{1.f, 0}, workspace,
+                              workspace_bytes, stream, "gdn_prefill_gated");
+}
+
+int gdn_prefill_fused(const void* q, const void* k, const void* v, const float* a, const float* b,
+                      const float* A_log, const float* dt_bias, const int32_t* cu_seqlens,
+                      const float* initial_state, void* out, float* final_state, int total_tokens, int num_seqs,
+                      int max_seqlen, int Hqk, int Hv, int dk, int dv, float scale, int qk_l2norm, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+    if (!front_ok(scale)) return GDN_ERR_SHAPE;
+    return prefill_front_impl(q, k, v, a, b, A_log, dt_bias, false, cu_seqlens, initial_state, out, final_state,
+                              total_tokens, num_seqs, max_seqlen, Hqk, Hv, dk, dv, QkFront{scale, qk_l2norm != 0},
+                              workspace, workspace_bytes, stream, "gdn_prefill_fused");
 }
 
 int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const float* g, const float* beta,
@@ -241,8 +288,9 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const flo
                                num_seqs, max_seqlen, Hqk, Hv, dk, dv, &nothing))
         return rc;
     if (nothing) return GDN_OK;
-    return cuda_status(prefill_recurrent_dispatch(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state,
-                                                  total_tokens, num_seqs, Hqk, Hv, nullptr, (cudaStream_t)stream),
+    return cuda_status(prefill_recurrent_dispatch(q, k, v, g, beta, nullptr, nullptr, cu_seqlens, initial_state, out,
+                                                  final_state, total_tokens, num_seqs, Hqk, Hv, nullptr,
+                                                  QkFront{1.f, 0}, (cudaStream_t)stream),
                        "gdn_prefill_recurrent");
 }
 

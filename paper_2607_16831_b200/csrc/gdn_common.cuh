@@ -51,6 +51,16 @@ __device__ __forceinline__ void raw_gates(float a, float b, float A_log, float d
     beta = 1.f / (1.f + __expf(-b));
 }
 
+// q/k front end of the fused entry points: with l2norm, q and k of a (token, head) are divided by
+// sqrt(sum of squares + kNormEps); q is then multiplied by scale.  Both enter every formula through
+// two per-token scalars, rq = scale / |q| and rk = 1 / |k|, so no normalised copy of q or k is made.
+struct QkFront {
+    float scale;
+    int l2norm;
+    __host__ __device__ bool active() const { return l2norm != 0 || scale != 1.f; }
+};
+constexpr float kNormEps = 1e-6f;
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Programmatic dependent launch.  A kernel launched with launch_pdl may be scheduled while the

@@ -66,7 +66,7 @@ cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v
                                      const int32_t* cu_seqlens, const float* initial_state,
                                      void* out, float* final_state, int total_tokens, int num_seqs,
                                      int max_seqlen, int Hqk, int Hv, void* workspace, size_t /*workspace_bytes*/,
-                                     bool allow_split, cudaStream_t st) {
+                                     bool allow_split, QkFront fr, cudaStream_t st) {
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     const WsLayout L = ws_layout(total_tokens, num_seqs, Hv, allow_split);
     // with few sequences the intra-chunk kernel builds the chunk table itself (one launch less)
@@ -79,7 +79,7 @@ cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v
             !make_map(&mv, v, total_tokens, Hv))
             return cudaErrorUnknown;
         e = launch_prefill_intra(mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv, no_prep ? cu_seqlens : nullptr, num_seqs,
-                                 total_tokens, st);
+                                 total_tokens, fr, st);
         if (e != cudaSuccess) return e;
         const int segs = choose_segments(L, num_seqs, Hv, max_seqlen);
         e = launch_prefill_chain(mq, mk, mv, initial_state, out, final_state, ws, L, num_seqs, Hqk, Hv, segs,
@@ -119,7 +119,8 @@ cudaError_t prefill_partial_dispatch(const void* q, const void* k, const void* v
         if (!make_map(&mq, q, total_tokens, Hqk) || !make_map(&mk, k, total_tokens, Hqk) ||
             !make_map(&mv, v, total_tokens, Hv))
             return cudaErrorUnknown;
-        e = launch_prefill_intra(mq, mk, g, beta, nullptr, nullptr, ws, L, Hqk, Hv, nullptr, num_seqs, total_tokens, st);
+        e = launch_prefill_intra(mq, mk, g, beta, nullptr, nullptr, ws, L, Hqk, Hv, nullptr, num_seqs, total_tokens,
+                                 QkFront{1.f, 0}, st);
         if (e != cudaSuccess) return e;
     } else {
         // no tensor to describe; every sequence is empty and the chain CTAs return before using the maps

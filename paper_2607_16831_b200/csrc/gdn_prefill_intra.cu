@@ -89,8 +89,8 @@ constexpr uint32_t IDG = IQ_LO;    // after MMA1: diagonal blocks of A^T, fp32 [
 constexpr uint32_t IBT2 = IQ_HI;   // after MMA1: B tiles of column block 2 (hi 4 KB | lo 4 KB)
 constexpr uint32_t IBT = 32768;    // B tiles of column blocks 0 and 1: [jb][hi|lo] x 4 KB               16 KB
 constexpr uint32_t IT2 = IBT;      // after the solve: T'' operand (bf16) [128][64]                       16 KB
-constexpr uint32_t IGAM = IBT + 16384;  // gam[2][64] | bet[2][64] | Gam[2][64] | cfP[2][64] | cfA[2][64] | alp[2][64] | tmp[4]
-constexpr uint32_t IBAR = IGAM + 12 * 64 * 4 + 64;
+constexpr uint32_t IGAM = IBT + 16384;  // gam[2][64] | bet[2][64] | Gam[2][64] | cfP[2][64] | cfA[2][64] | alp[2][64] | rq[64] | rk[64] | tmp[4]
+constexpr uint32_t IBAR = IGAM + 14 * 64 * 4 + 64;
 constexpr uint32_t kIntraSmem = IBAR + 64 + 1024;
 // tensor-memory columns: [QK^T ; KK^T] first, then the solve's operands, then the W accumulator
 constexpr uint32_t ITM_D1 = 0, ITM_YHI = 0, ITM_YLO = 32, ITM_ACC = 64, ITM_D2 = 0, ITM_COLS = 128;
@@ -99,12 +99,18 @@ __device__ __forceinline__ uint32_t intra_btile(int jb, int lo) {  // byte offse
     return (jb == 2 ? IBT2 : IBT + (uint32_t)jb * 8192u) + (uint32_t)lo * 4096u;
 }
 
+// FRONT: the fused entry points' q/k front end (QkFront).  q and k stay as they are in shared memory and
+// in the products; the per-token factors rq_i = scale / |q_i| and rk_j = 1 / |k_j| go into the
+// coefficients instead: A_mj gets rk_m rk_j, P_ij gets rq_i rk_j, the K-side diagonal of W and the
+// state update's e_j get rk_j, the output scaling Gamma_i gets rq_i.  The kernels after this one
+// see nothing of it.
+template <bool FRONT>
 __global__ void __launch_bounds__(kIntraThreads, 4)
 gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                          const float* __restrict__ g, const float* __restrict__ beta,
                          const float* __restrict__ A_log, const float* __restrict__ dt_bias,
                          uint8_t* __restrict__ ws, WsLayout L, int Hqk, int Hv, const int32_t* __restrict__ cu,
-                         int num_seqs, int total_tokens) {
+                         int num_seqs, int total_tokens, QkFront fr) {
     const int c = blockIdx.x;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     int t0, len;
@@ -183,7 +189,9 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     float* cfP = gam + 384;  // exp(gamma_{last column of j's 16-block} - gamma_j)
     float* cfA = gam + 512;  // beta_m exp(gamma_m - gamma_{first row of m's 16-block})
     float* alp = gam + 640;  // per-token decay exp(g_t) = exp(gamma_t - gamma_{t-1})
-    float* tmp = gam + 768;
+    float* rq = gam + 768;   // FRONT only: scale / |q_i|
+    float* rk = gam + 832;   // FRONT only: 1 / |k_j|
+    float* tmp = gam + 896;
     uint64_t* bar_load = reinterpret_cast<uint64_t*>(smem + IBAR);
     uint64_t* bar_mma1 = bar_load + 1;
     uint64_t* bar_mma2 = bar_load + 2;
@@ -252,8 +260,8 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         cfP[tid] = __expf(gam[(tid & ~15) | 15] - x);
         cfA[tid] = b * __expf(x - gam[tid & ~15]);
     }
+    if (FRONT || warp == 0) ok = mbar_wait_all(bar_load, 0, abort_flag);
     if (warp == 0) {
-        ok = mbar_wait_all(bar_load, 0, abort_flag);
         if (ok) {
             tc_fence_after_sync();
             constexpr uint32_t ID1 = umma_idesc_bf16(128, 64, false, false, false);
@@ -264,9 +272,39 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) umma_bf16_ss_warp(tmem_base + ITM_D1, dA1 + ks * 2, dB1 + ks * 2, ID1, 1);
             umma_commit_warp(bar_mma1);
-            ok = mbar_wait_all(bar_mma1, 0, abort_flag);  // only this warp polls; the others park at the barrier
         }
     }
+    if constexpr (FRONT) {
+        // while MMA1 runs: thread r < 64 takes row r of Q, thread 64 + r row r of K.  A row is 128 bytes
+        // in each of the two tiles; the 128-byte swizzle only permutes its 16-byte pieces, and a sum
+        // over all of them does not care (pieces taken in a rotated order to spread the banks).
+        float f = (tid < 64) ? fr.scale : 1.f;
+        if (fr.l2norm && ok) {
+            const uint8_t* lo = smem + (tid < 64 ? IQ_LO : IK_LO) + (uint32_t)(tid & 63) * 128u;
+            const uint8_t* hi = smem + (tid < 64 ? IQ_HI : IK_HI) + (uint32_t)(tid & 63) * 128u;
+            float ss = 0.f;
+#pragma unroll
+            for (int cc = 0; cc < 8; ++cc) {
+                const int ch = (cc + tid) & 7;
+                const uint4 a = *reinterpret_cast<const uint4*>(lo + ch * 16);
+                const uint4 b = *reinterpret_cast<const uint4*>(hi + ch * 16);
+                const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    float x0, x1;
+                    unpack_bf16x2(w[u], x0, x1);
+                    ss = fmaf(x0, x0, ss);
+                    ss = fmaf(x1, x1, ss);
+                }
+            }
+            f *= rsqrtf(ss + kNormEps);
+        }
+        rq[tid] = f;  // rq and rk are adjacent: thread 64 + r writes rk[r]
+        __syncthreads();
+        cfP[tid] *= rk[i];
+        cfA[tid] *= rk[i];
+    }
+    if (warp == 0 && ok) ok = mbar_wait_all(bar_mma1, 0, abort_flag);  // only this warp polls; the others park at the barrier
     ok = __syncthreads_and(ok);
     GDN_ISTAMP(1);
     if (ok) {
@@ -274,8 +312,9 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         // per-token scalars of this thread's (head, row)
         if (head_ok) {
             float* wsS = reinterpret_cast<float*>(ws + L.off_scal + ((size_t)c * Hv + h) * kScalBytes);
-            wsS[i] = Gam[tid];
-            wsS[64 + i] = __expf(gam[hh * 64 + len - 1] - gam[tid]);
+            wsS[i] = FRONT ? Gam[tid] * rq[i] : Gam[tid];
+            const float e_i = __expf(gam[hh * 64 + len - 1] - gam[tid]);
+            wsS[64 + i] = FRONT ? e_i * rk[i] : e_i;
             if (i == 0) wsS[128] = Gam[hh * 64 + len - 1];
         }
         // ---- phase A, sixteen columns at a time (rolled: long straight-line code runs at
@@ -309,7 +348,8 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         // diagonal block for one half of the warp take the per-element form for all 32 lanes.
                         const int wb2 = (row >> 5) * 2;
                         if (q4 < wb2) {
-                            const float rf = (row < len) ? __expf(gi - gam[e * 64 + q4 * 16 + 15]) : 0.f;
+                            float rf = (row < len) ? __expf(gi - gam[e * 64 + q4 * 16 + 15]) : 0.f;
+                            if constexpr (FRONT) rf *= rq[row];
                             const float* cf = cfP + e * 64 + q4 * 16;
 #pragma unroll
                             for (int jl = 0; jl < 16; ++jl) pv[jl] = __uint_as_float(r[jl]) * (rf * cf[jl]);
@@ -319,10 +359,14 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                             // is <= 1, so nothing can overflow): acc = exp(gamma_i - gamma_j) once j <= i
                             float acc = __expf(fminf(gi - gm[15], 0.f));  // 1 for rows inside the block
                             const float* al = alp + e * 64 + q4 * 16;
+                            const float rqi = FRONT ? rq[row] : 1.f;
 #pragma unroll
                             for (int jl = 15; jl >= 0; --jl) {
                                 const bool on = (q4 * 16 + jl <= row) && (row < len);
-                                pv[jl] = on ? __uint_as_float(r[jl]) * acc : 0.f;
+                                if constexpr (FRONT)
+                                    pv[jl] = on ? __uint_as_float(r[jl]) * (acc * (rqi * rk[q4 * 16 + jl])) : 0.f;
+                                else
+                                    pv[jl] = on ? __uint_as_float(r[jl]) * acc : 0.f;
                                 acc = on ? acc * al[jl] : acc;
                             }
                         } else {
@@ -342,15 +386,19 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                             const float* bm = bet + e * 64 + q4 * 16;
                             // exp(gamma_m - gamma_j), m > j, as the running product of the per-token decays
                             const float* al = alp + e * 64 + q4 * 16;
-                            float acc = 1.f;
+                            float acc = FRONT ? rk[row] : 1.f;
 #pragma unroll
                             for (int ml = 0; ml < 16; ++ml) {
                                 const bool on = q4 * 16 + ml > row;
                                 acc = on ? acc * al[ml] : acc;
-                                a[ml] = on ? bm[ml] * acc * __uint_as_float(r[ml]) : 0.f;
+                                if constexpr (FRONT)
+                                    a[ml] = on ? (bm[ml] * rk[q4 * 16 + ml]) * acc * __uint_as_float(r[ml]) : 0.f;
+                                else
+                                    a[ml] = on ? bm[ml] * acc * __uint_as_float(r[ml]) : 0.f;
                             }
                         } else {
-                            const float rf = __expf(gam[e * 64 + q4 * 16] - gi);
+                            float rf = __expf(gam[e * 64 + q4 * 16] - gi);
+                            if constexpr (FRONT) rf *= rk[row];
                             const float* cf = cfA + e * 64 + q4 * 16;
 #pragma unroll
                             for (int ml = 0; ml < 16; ++ml) a[ml] = (rf * cf[ml]) * __uint_as_float(r[ml]);
@@ -457,7 +505,10 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     const float a0 = z[c16 >> 1][(c16 & 1) * 8 + q2 * 2] * bt[j];
                     const float a1 = z[c16 >> 1][(c16 & 1) * 8 + q2 * 2 + 1] * bt[j + 1];
                     split_bf16x2(a0, a1, h1[q2], l1[q2]);
-                    h2[q2] = pack_bf16x2(a0 * Gm[j], a1 * Gm[j + 1]);
+                    if constexpr (FRONT)
+                        h2[q2] = pack_bf16x2(a0 * (Gm[j] * rk[j]), a1 * (Gm[j + 1] * rk[j + 1]));
+                    else
+                        h2[q2] = pack_bf16x2(a0 * Gm[j], a1 * Gm[j + 1]);
                 }
                 if (head_ok) {
                     *reinterpret_cast<uint4*>(wsA + swz(i, c16)) = make_uint4(h1[0], h1[1], h1[2], h1[3]);
@@ -528,17 +579,26 @@ cudaError_t launch_prefill_prep(const int32_t* cu_seqlens, int num_seqs, int tot
 
 cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, const float* g, const float* beta,
                                  const float* A_log, const float* dt_bias, uint8_t* ws, const WsLayout& L, int Hqk,
-                                 int Hv, const int32_t* cu_if_no_table, int num_seqs, int total_tokens,
+                                 int Hv, const int32_t* cu_if_no_table, int num_seqs, int total_tokens, QkFront fr,
                                  cudaStream_t st) {
     static bool attr_done[64];
     if (cudaError_t e = set_attrs_once(attr_done, [] {
-            return cudaFuncSetAttribute(gdn_prefill_intra_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kIntraSmem);
+            cudaError_t e2 = cudaFuncSetAttribute(gdn_prefill_intra_kernel<false>,
+                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, kIntraSmem);
+            if (e2 == cudaSuccess)
+                e2 = cudaFuncSetAttribute(gdn_prefill_intra_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          kIntraSmem);
+            return e2;
         }))
         return e;
     const int G = Hv / Hqk;
     dim3 grid(L.nc_max, Hqk * ((G + 1) / 2));
-    gdn_prefill_intra_kernel<<<grid, kIntraThreads, kIntraSmem, st>>>(mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv,
-                                                                      cu_if_no_table, num_seqs, total_tokens);
+    if (fr.active())
+        gdn_prefill_intra_kernel<true><<<grid, kIntraThreads, kIntraSmem, st>>>(
+            mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv, cu_if_no_table, num_seqs, total_tokens, fr);
+    else
+        gdn_prefill_intra_kernel<false><<<grid, kIntraThreads, kIntraSmem, st>>>(
+            mq, mk, g, beta, A_log, dt_bias, ws, L, Hqk, Hv, cu_if_no_table, num_seqs, total_tokens, fr);
     return cudaGetLastError();
 }
 

@@ -10,7 +10,7 @@ cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v
                                      const int32_t* cu_seqlens, const float* initial_state,
                                      void* out, float* final_state, int total_tokens, int num_seqs,
                                      int max_seqlen, int Hqk, int Hv, void* workspace, size_t workspace_bytes,
-                                     bool allow_split, cudaStream_t st);
+                                     bool allow_split, QkFront fr, cudaStream_t st);
 }  // namespace gdn
 
 // The scratch itself.  Every device that loads the library carries these bytes until the
@@ -57,6 +57,7 @@ extern "C" int gdn_prefill_static(const void* q, const void* k, const void* v, c
     }
     cudaError_t e = prefill_chunked_dispatch(q, k, v, g, beta, nullptr, nullptr, cu_seqlens, initial_state, out, final_state,
                                              total_tokens, num_seqs, max_seqlen, Hqk, Hv, g_static_scratch_addr[dev],
-                                             (size_t)GDN_PREFILL_STATIC_SCRATCH_BYTES, false, (cudaStream_t)stream);
+                                             (size_t)GDN_PREFILL_STATIC_SCRATCH_BYTES, false, QkFront{1.f, 0},
+                                             (cudaStream_t)stream);
     return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }

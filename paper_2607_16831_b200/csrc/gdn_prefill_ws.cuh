@@ -89,7 +89,7 @@ cudaError_t launch_prefill_prep(const int32_t* cu_seqlens, int num_seqs, int tot
 constexpr int kMaxSeqsWithoutPrep = 8;
 cudaError_t launch_prefill_intra(const CUtensorMap& mq, const CUtensorMap& mk, const float* g, const float* beta,
                                  const float* A_log, const float* dt_bias, uint8_t* ws, const WsLayout& L, int Hqk,
-                                 int Hv, const int32_t* cu_if_no_table, int num_seqs, int total_tokens,
+                                 int Hv, const int32_t* cu_if_no_table, int num_seqs, int total_tokens, QkFront fr,
                                  cudaStream_t st);
 // Destinations of the chain kernel's partial mode (gdn_prefill_partial): all NULL = normal mode.
 struct ChainPartial {

@@ -63,6 +63,18 @@ def test_host_side_argument_checks(gdn):
     a = list(args); a[0] = odd
     assert L.gdn_prefill(*a, 100, 2, 60, 16, 32, 128, 128, fake, 1 << 30, None) == 5
     assert L.gdn_prefill_recurrent(*args, 100, 2, 101, 16, 32, 128, 128, None) == 2
+    # fused front end
+    assert L.gdn_decode_fused(fake, fake, fake, fake, fake, None, fake, fake, fake, fake, 2, 16, 32, 128, 128, 1.0, 1, None) == 1
+    assert L.gdn_decode_fused(fake, fake, fake, fake, fake, None, None, fake, fake, fake, 2, 16, 32, 128, 128,
+                              float("inf"), 1, None) == 2
+    assert L.gdn_decode_fused(fake, fake, fake, fake, fake, None, None, fake, fake, fake, 0, 16, 32, 128, 128, 1.0, 1, None) == 0
+    fa = [fake] * 11
+    assert L.gdn_prefill_fused(*fa, 100, 2, 60, 16, 32, 128, 128, float("nan"), 0, fake, 1 << 30, None) == 2
+    a = list(fa); a[5] = None   # A_log without dt_bias
+    assert L.gdn_prefill_fused(*a, 100, 2, 60, 16, 32, 128, 128, 1.0, 1, fake, 1 << 30, None) == 1
+    a = list(fa); a[1] = odd
+    assert L.gdn_prefill_fused(*a, 100, 2, 60, 16, 32, 128, 128, 1.0, 1, fake, 1 << 30, None) == 5
+    assert L.gdn_prefill_fused(*fa, 0, 0, 0, 16, 32, 128, 128, 1.0, 1, None, 0, None) == 0
     # sequence-parallel building blocks
     pa = [fake] * 10
     assert L.gdn_prefill_partial(*pa, 0, 0, 0, 16, 32, 128, 128, None, 0, None) == 0
