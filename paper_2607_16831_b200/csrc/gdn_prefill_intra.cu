@@ -95,6 +95,15 @@ constexpr uint32_t kIntraSmem = IBAR + 64 + 1024;
 // tensor-memory columns: [QK^T ; KK^T] first, then the solve's operands, then the W accumulator
 constexpr uint32_t ITM_D1 = 0, ITM_YHI = 0, ITM_YLO = 32, ITM_ACC = 64, ITM_D2 = 0, ITM_COLS = 128;
 
+// sixteen consecutive floats of a coefficient table (64-byte aligned) as four 16-byte loads
+__device__ __forceinline__ void ld16(const float* p, float (&x)[16]) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const float4 t = reinterpret_cast<const float4*>(p)[q];
+        x[4 * q] = t.x; x[4 * q + 1] = t.y; x[4 * q + 2] = t.z; x[4 * q + 3] = t.w;
+    }
+}
+
 __device__ __forceinline__ uint32_t intra_btile(int jb, int lo) {  // byte offset of B tile (jb, hi/lo)
     return (jb == 2 ? IBT2 : IBT + (uint32_t)jb * 8192u) + (uint32_t)lo * 4096u;
 }
@@ -350,7 +359,8 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         if (q4 < wb2) {
                             float rf = (row < len) ? __expf(gi - gam[e * 64 + q4 * 16 + 15]) : 0.f;
                             if constexpr (FRONT) rf *= rq[row];
-                            const float* cf = cfP + e * 64 + q4 * 16;
+                            float cf[16];
+                            ld16(cfP + e * 64 + q4 * 16, cf);
 #pragma unroll
                             for (int jl = 0; jl < 16; ++jl) pv[jl] = __uint_as_float(r[jl]) * (rf * cf[jl]);
                         } else if (q4 <= wb2 + 1) {
@@ -358,13 +368,19 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                             // of the per-token decays (one exp per row instead of sixteen; every factor
                             // is <= 1, so nothing can overflow): acc = exp(gamma_i - gamma_j) once j <= i
                             float acc = __expf(fminf(gi - gm[15], 0.f));  // 1 for rows inside the block
-                            const float* al = alp + e * 64 + q4 * 16;
-                            const float rqi = FRONT ? rq[row] : 1.f;
+                            float al[16], kq[16];
+                            ld16(alp + e * 64 + q4 * 16, al);
+                            if constexpr (FRONT) {
+                                ld16(rk + q4 * 16, kq);
+                                const float rqi = rq[row];
+#pragma unroll
+                                for (int x = 0; x < 16; ++x) kq[x] *= rqi;
+                            }
 #pragma unroll
                             for (int jl = 15; jl >= 0; --jl) {
                                 const bool on = (q4 * 16 + jl <= row) && (row < len);
                                 if constexpr (FRONT)
-                                    pv[jl] = on ? __uint_as_float(r[jl]) * (acc * (rqi * rk[q4 * 16 + jl])) : 0.f;
+                                    pv[jl] = on ? __uint_as_float(r[jl]) * (acc * kq[jl]) : 0.f;
                                 else
                                     pv[jl] = on ? __uint_as_float(r[jl]) * acc : 0.f;
                                 acc = on ? acc * al[jl] : acc;
@@ -373,40 +389,46 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
                             for (int jl = 0; jl < 16; ++jl) pv[jl] = 0.f;
                         }
+                        {   // the sixteen columns are two adjacent 16-byte chunks of the row: one 32-byte store
+                            uint32_t pk[8];
 #pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            uint32_t pk[4];
-#pragma unroll
-                            for (int q2 = 0; q2 < 4; ++q2) pk[q2] = pack_bf16x2(pv[half * 8 + q2 * 2], pv[half * 8 + q2 * 2 + 1]);
-                            *reinterpret_cast<uint4*>(wsP + swz(row, q4 * 2 + half)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            for (int q2 = 0; q2 < 8; ++q2) pk[q2] = pack_bf16x2(pv[q2 * 2], pv[q2 * 2 + 1]);
+                            st_swizzled_pair(wsP, (uint32_t)row, (uint32_t)q4, make_uint4(pk[0], pk[1], pk[2], pk[3]),
+                                             make_uint4(pk[4], pk[5], pk[6], pk[7]));
                         }
                     } else if (q4 >= jb_own) {
                         float a[16];
                         if (q4 == jb_own) {
-                            const float* bm = bet + e * 64 + q4 * 16;
+                            float bm[16], al[16];
+                            ld16(bet + e * 64 + q4 * 16, bm);
                             // exp(gamma_m - gamma_j), m > j, as the running product of the per-token decays
-                            const float* al = alp + e * 64 + q4 * 16;
+                            ld16(alp + e * 64 + q4 * 16, al);
                             float acc = FRONT ? rk[row] : 1.f;
+                            if constexpr (FRONT) {
+                                float k16[16];
+                                ld16(rk + q4 * 16, k16);
+#pragma unroll
+                                for (int x = 0; x < 16; ++x) bm[x] *= k16[x];
+                            }
 #pragma unroll
                             for (int ml = 0; ml < 16; ++ml) {
                                 const bool on = q4 * 16 + ml > row;
                                 acc = on ? acc * al[ml] : acc;
-                                if constexpr (FRONT)
-                                    a[ml] = on ? (bm[ml] * rk[q4 * 16 + ml]) * acc * __uint_as_float(r[ml]) : 0.f;
-                                else
-                                    a[ml] = on ? bm[ml] * acc * __uint_as_float(r[ml]) : 0.f;
+                                a[ml] = on ? bm[ml] * acc * __uint_as_float(r[ml]) : 0.f;
                             }
                         } else {
                             float rf = __expf(gam[e * 64 + q4 * 16] - gi);
                             if constexpr (FRONT) rf *= rk[row];
-                            const float* cf = cfA + e * 64 + q4 * 16;
+                            float cf[16];
+                            ld16(cfA + e * 64 + q4 * 16, cf);
 #pragma unroll
                             for (int ml = 0; ml < 16; ++ml) a[ml] = (rf * cf[ml]) * __uint_as_float(r[ml]);
                         }
                         if (q4 == jb_own) {
-                            float4* dg = reinterpret_cast<float4*>(smem + IDG) + ((e * 4 + jb_own) * 16 + (row & 15)) * 4;
+                            // stored by row m: the solve reads, for one m, the run of columns j < m as float4s
+                            float* dg = reinterpret_cast<float*>(smem + IDG) + (e * 4 + jb_own) * 256 + (row & 15);
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) dg[q] = make_float4(a[4 * q], a[4 * q + 1], a[4 * q + 2], a[4 * q + 3]);
+                            for (int ml = 0; ml < 16; ++ml) dg[ml * 16] = a[ml];
                         } else {
                             const uint32_t n = (uint32_t)(e * 16 + (row & 15));
 #pragma unroll
@@ -450,12 +472,20 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
             // diagonal block, column by column from the right: once z_mm is known its contribution is
             // pushed to every column left of it (independent FMAs, no long chain)
-            const float* dg = reinterpret_cast<const float*>(smem + IDG) + (hh * 4 + jb) * 256;
+            // (entries at and right of the diagonal are stored as zeros, so whole float4s are applied)
+            const float4* dg = reinterpret_cast<const float4*>(smem + IDG) + (hh * 4 + jb) * 64;
 #pragma unroll
             for (int mm = 15; mm >= 0; --mm) {
-                z[jb][mm] = rhs[mm];
+                const float zm = rhs[mm];
+                z[jb][mm] = zm;
 #pragma unroll
-                for (int jj = 0; jj < mm; ++jj) rhs[jj] = fmaf(-dg[jj * 16 + mm], z[jb][mm], rhs[jj]);
+                for (int q = 0; q < (mm + 3) / 4; ++q) {
+                    const float4 d = dg[mm * 4 + q];
+                    rhs[4 * q + 0] = fmaf(-d.x, zm, rhs[4 * q + 0]);
+                    rhs[4 * q + 1] = fmaf(-d.y, zm, rhs[4 * q + 1]);
+                    rhs[4 * q + 2] = fmaf(-d.z, zm, rhs[4 * q + 2]);
+                    rhs[4 * q + 3] = fmaf(-d.w, zm, rhs[4 * q + 3]);
+                }
             }
             GDN_ISTAMP(3 + 2 * (3 - jb));
             if (jb > 0) {
@@ -490,37 +520,53 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 GDN_ISTAMP(4 + 2 * (3 - jb));
             }
         }
+        // The images that go to the workspace (T' hi, T' lo, W) are row-major with 128-byte rows and a thread
+        // owns a row, so a direct 16-byte store instruction would touch 32 different lines.  They are built
+        // in shared memory instead (conflict-free with the swizzle) and leave as bulk copies: T' hi now, over
+        // the diagonal blocks and the B tiles of column block 2 (hence the barrier: the last solve step of
+        // other warps may still be reading the diagonal blocks); T' lo and W after MMA2, when the rest is free.
+        uint8_t* wsA = ws + L.off_A + ((size_t)c * Hv + h) * kABytes;
+        uint8_t* stHi = smem + (hh ? IBT2 : IDG);
+        __syncthreads();
         if (ok) {
-            // ---- T' = T diag(beta) -> workspace (bf16 hi + lo); T'' = T' diag(Gamma) -> smem A operand
-            //      (bf16), over the B tiles, which the last step's MMAs have finished reading
-            uint8_t* wsA = ws + L.off_A + ((size_t)c * Hv + h) * kABytes;
+            // ---- T' = T diag(beta) (bf16 hi here, lo below); T'' = T' diag(Gamma) -> smem A operand (bf16),
+            //      over the B tiles, which the last step's MMAs have finished reading
             const float* bt = bet + hh * 64;
             const float* Gm = Gam + hh * 64;
 #pragma unroll
-            for (int c16 = 0; c16 < 8; ++c16) {
-                uint32_t h1[4], l1[4], h2[4];
+            for (int cp = 0; cp < 4; ++cp) {  // sixteen columns at a time
+                uint32_t h1[8], l1[8], h2[8];
+                float b16[16], G16[16];
+                ld16(bt + cp * 16, b16);
+                ld16(Gm + cp * 16, G16);
+                if constexpr (FRONT) {
+                    float k16[16];
+                    ld16(rk + cp * 16, k16);
 #pragma unroll
-                for (int q2 = 0; q2 < 4; ++q2) {
-                    const int j = c16 * 8 + q2 * 2;
-                    const float a0 = z[c16 >> 1][(c16 & 1) * 8 + q2 * 2] * bt[j];
-                    const float a1 = z[c16 >> 1][(c16 & 1) * 8 + q2 * 2 + 1] * bt[j + 1];
+                    for (int x = 0; x < 16; ++x) G16[x] *= k16[x];
+                }
+#pragma unroll
+                for (int q2 = 0; q2 < 8; ++q2) {
+                    const float a0 = z[cp][q2 * 2] * b16[q2 * 2];
+                    const float a1 = z[cp][q2 * 2 + 1] * b16[q2 * 2 + 1];
                     split_bf16x2(a0, a1, h1[q2], l1[q2]);
-                    if constexpr (FRONT)
-                        h2[q2] = pack_bf16x2(a0 * (Gm[j] * rk[j]), a1 * (Gm[j + 1] * rk[j + 1]));
-                    else
-                        h2[q2] = pack_bf16x2(a0 * Gm[j], a1 * Gm[j + 1]);
+                    h2[q2] = pack_bf16x2(a0 * G16[q2 * 2], a1 * G16[q2 * 2 + 1]);
                 }
-                if (head_ok) {
-                    *reinterpret_cast<uint4*>(wsA + swz(i, c16)) = make_uint4(h1[0], h1[1], h1[2], h1[3]);
-                    *reinterpret_cast<uint4*>(wsA + 8192 + swz(i, c16)) = make_uint4(l1[0], l1[1], l1[2], l1[3]);
-                }
-                *reinterpret_cast<uint4*>(smem + IT2 + swz(tid, c16)) = make_uint4(h2[0], h2[1], h2[2], h2[3]);
+                *reinterpret_cast<uint4*>(stHi + swz(i, 2 * cp)) = make_uint4(h1[0], h1[1], h1[2], h1[3]);
+                *reinterpret_cast<uint4*>(stHi + swz(i, 2 * cp + 1)) = make_uint4(h1[4], h1[5], h1[6], h1[7]);
+                *reinterpret_cast<uint4*>(smem + IT2 + swz(tid, 2 * cp)) = make_uint4(h2[0], h2[1], h2[2], h2[3]);
+                *reinterpret_cast<uint4*>(smem + IT2 + swz(tid, 2 * cp + 1)) = make_uint4(h2[4], h2[5], h2[6], h2[7]);
             }
             fence_proxy_async_smem();
             tc_fence_before_sync();
         }
         __syncthreads();
         GDN_ISTAMP(11);
+        const bool storer = ok && i == 0 && head_ok;  // threads 0 and 64: one per head
+        if (storer) {
+            bulk_store(wsA, stHi, 8192);
+            bulk_store_commit();
+        }
         // ---- MMA2: W (both heads) = [T''_a ; T''_b] K, K read MN-major from the TMA tiles
         if (ok && warp == 0) {
             tc_fence_after_sync();
@@ -532,30 +578,55 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             umma_commit_warp(bar_mma2);
             ok = mbar_wait_all(bar_mma2, 0, abort_flag);
         }
+        if (storer) bulk_store_wait_read();  // the staging of T' hi is written again below
         ok = __syncthreads_and(ok);
         GDN_ISTAMP(12);
+        if (ok) {
+            // ---- T' lo (the bf16 remainder, recomputed from the solve's registers) -> staging over the T''
+            //      operand, which MMA2 has finished reading
+            uint8_t* stLo = smem + IT2 + (uint32_t)hh * 8192u;
+            const float* bt = bet + hh * 64;
+#pragma unroll
+            for (int cp = 0; cp < 4; ++cp) {
+                uint32_t h1[8], l1[8];
+                float b16[16];
+                ld16(bt + cp * 16, b16);
+#pragma unroll
+                for (int q2 = 0; q2 < 8; ++q2)
+                    split_bf16x2(z[cp][q2 * 2] * b16[q2 * 2], z[cp][q2 * 2 + 1] * b16[q2 * 2 + 1], h1[q2], l1[q2]);
+                *reinterpret_cast<uint4*>(stLo + swz(i, 2 * cp)) = make_uint4(l1[0], l1[1], l1[2], l1[3]);
+                *reinterpret_cast<uint4*>(stLo + swz(i, 2 * cp + 1)) = make_uint4(l1[4], l1[5], l1[6], l1[7]);
+            }
+        }
     }
     if (ok) {
         tc_fence_after_sync();
-        // ---- W row i of head h -> workspace (K-major B operand image: two [64][64] tiles)
-        uint8_t* wsW = ws + L.off_A + ((size_t)c * Hv + h) * kABytes + 16384;
+        // ---- W row i of head h (K-major B operand image: two [64][64] tiles) -> staging over the q/k tiles
+        uint8_t* stW = smem + (uint32_t)hh * 16384u;
 #pragma unroll 1
         for (int b = 0; b < 4; ++b) {
             uint32_t r[32];
             tmem_ld32(lane_addr + ITM_D2 + b * 32, r);
             tmem_ld_wait();
-            if (head_ok) {
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-                    uint4 o;
-                    o.x = pack_bf16x2(__uint_as_float(r[cc * 8 + 0]), __uint_as_float(r[cc * 8 + 1]));
-                    o.y = pack_bf16x2(__uint_as_float(r[cc * 8 + 2]), __uint_as_float(r[cc * 8 + 3]));
-                    o.z = pack_bf16x2(__uint_as_float(r[cc * 8 + 4]), __uint_as_float(r[cc * 8 + 5]));
-                    o.w = pack_bf16x2(__uint_as_float(r[cc * 8 + 6]), __uint_as_float(r[cc * 8 + 7]));
-                    *reinterpret_cast<uint4*>(wsW + (b >> 1) * 8192 + swz(i, (b & 1) * 4 + cc)) = o;
-                }
+            for (int cc = 0; cc < 4; ++cc) {
+                uint4 o;
+                o.x = pack_bf16x2(__uint_as_float(r[cc * 8 + 0]), __uint_as_float(r[cc * 8 + 1]));
+                o.y = pack_bf16x2(__uint_as_float(r[cc * 8 + 2]), __uint_as_float(r[cc * 8 + 3]));
+                o.z = pack_bf16x2(__uint_as_float(r[cc * 8 + 4]), __uint_as_float(r[cc * 8 + 5]));
+                o.w = pack_bf16x2(__uint_as_float(r[cc * 8 + 6]), __uint_as_float(r[cc * 8 + 7]));
+                *reinterpret_cast<uint4*>(stW + (b >> 1) * 8192 + swz(i, (b & 1) * 4 + cc)) = o;
             }
         }
+        fence_proxy_async_smem();
+    }
+    __syncthreads();
+    if (ok && i == 0 && head_ok) {
+        uint8_t* wsA = ws + L.off_A + ((size_t)c * Hv + h) * kABytes;
+        bulk_store(wsA + 8192, smem + IT2 + (uint32_t)hh * 8192u, 8192);  // T' lo
+        bulk_store(wsA + 16384, smem + (uint32_t)hh * 16384u, 16384);     // W
+        bulk_store_commit();
+        bulk_store_wait_read();  // shared memory must outlive the copy's reads
     }
 
     GDN_ISTAMP(13);

@@ -146,6 +146,33 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
         : "memory");
 }
+// One 32-byte global store (st.global.v8: sm_100 and later); the address must be 32-byte aligned.
+__device__ __forceinline__ void st_global_v8(void* p, uint4 lo, uint4 hi) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w)
+                 : "memory");
+}
+// The two 16-byte chunks 2m and 2m + 1 of row r of a 128-byte-swizzled image share one aligned 32-byte
+// sector (the swizzle XORs the chunk index with r % 8: for odd r the two swap places).
+__device__ __forceinline__ void st_swizzled_pair(uint8_t* image, uint32_t r, uint32_t m, uint4 c_even, uint4 c_odd) {
+    uint8_t* p = image + r * 128u + (((2u * m) ^ (r & 6u)) * 16u);
+    if (r & 1u)
+        st_global_v8(p, c_odd, c_even);
+    else
+        st_global_v8(p, c_even, c_odd);
+}
+
+// 1-D bulk copy shared -> global (same alignment rules).  The copies of a thread form groups:
+// bulk_store_commit closes the group, bulk_store_wait_read returns once every committed group of
+// this thread has finished READING shared memory (the data may still be on its way to global
+// memory; it is visible to later kernels like any other write of this one).
+__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(reinterpret_cast<uint64_t>(gdst)), "r"(smem_u32(smem_src)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
