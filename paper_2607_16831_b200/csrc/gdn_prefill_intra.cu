@@ -460,6 +460,13 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         constexpr uint32_t IDS = umma_idesc_bf16(128, 32, false, false, false);
 #pragma unroll
         for (int jb = 3; jb >= 0; --jb) {
+            // T is lower triangular: a warp whose 32 rows all lie above column block jb (rows 0-31 of a head
+            // for blocks 2 and 3) has nothing but zeros there and skips the block's loads and arithmetic
+            const bool dead = jb > 2 * (warp & 1) + 1;
+            if (dead) {
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) z[jb][jj] = 0.f;
+            } else {
             float rhs[16];
 #pragma unroll
             for (int jj = 0; jj < 16; ++jj) rhs[jj] = ((16 * jb + jj) == i) ? 1.f : 0.f;
@@ -486,6 +493,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     rhs[4 * q + 2] = fmaf(-d.z, zm, rhs[4 * q + 2]);
                     rhs[4 * q + 3] = fmaf(-d.w, zm, rhs[4 * q + 3]);
                 }
+            }
             }
             GDN_ISTAMP(3 + 2 * (3 - jb));
             if (jb > 0) {
