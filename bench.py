@@ -34,9 +34,9 @@ TOKEN_BYTES_PER_ITEM = 2 * 16 * 128 * 2 + 2 * 32 * 128 * 2 + 2 * 32 * 4   # q,k 
 PREFILL_BYTES_PER_TOKEN = 24832                          # q 4096 + k 4096 + v 8192 + out 8192 + g,beta 256
 PREFILL_FLOPS_PER_TOKEN = 5.77e6                         # 11.53 MFLOP per (chunk, value head) / 64 * 32
 # DRAM bytes per decode launch at B = 64 from the committed ncu capture
-# (profiles/decode_b64_ncu.md): 135.29 MB read + 79.69 MB written inside the launch window (the write-back
+# (profiles/decode_b64_ncu.md): 135.32 MB read + 82.30 MB written inside the launch window (the write-back
 # L2 still holds the tail of the 134 MB output when the kernel ends).
-DECODE_B64_DRAM_TRAFFIC = 218.03e6
+DECODE_B64_DRAM_TRAFFIC = 217.62e6
 
 
 def load_peaks():
