@@ -269,8 +269,8 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         cfP[tid] = __expf(gam[(tid & ~15) | 15] - x);
         cfA[tid] = b * __expf(x - gam[tid & ~15]);
     }
-    if (FRONT || warp == 0) ok = mbar_wait_all(bar_load, 0, abort_flag);
     if (warp == 0) {
+        ok = mbar_wait_all(bar_load, 0, abort_flag);
         if (ok) {
             tc_fence_after_sync();
             constexpr uint32_t ID1 = umma_idesc_bf16(128, 64, false, false, false);
@@ -287,7 +287,9 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         // while MMA1 runs: thread r < 64 takes row r of Q, thread 64 + r row r of K.  A row is 128 bytes
         // in each of the two tiles; the 128-byte swizzle only permutes its 16-byte pieces, and a sum
         // over all of them does not care (pieces taken in a rotated order to spread the banks).
+        // (only warp 0 polls the load barrier: the others learn of the tiles through the CTA barrier)
         float f = (tid < 64) ? fr.scale : 1.f;
+        if (fr.l2norm) ok = __syncthreads_and(ok);
         if (fr.l2norm && ok) {
             const uint8_t* lo = smem + (tid < 64 ? IQ_LO : IK_LO) + (uint32_t)(tid & 63) * 128u;
             const uint8_t* hi = smem + (tid < 64 ? IQ_HI : IK_HI) + (uint32_t)(tid & 63) * 128u;

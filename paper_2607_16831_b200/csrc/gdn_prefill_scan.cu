@@ -83,6 +83,7 @@ gdn_prefill_combine_kernel(ScanArgs A, int Hv, int nbuf) {
         mbar_fence_init();
         if (run_chunks(1) > 0) fetch_P(1);
     }
+    __syncthreads();  // the barriers and the abort flag are set before anybody reads them (the loop below may run zero times)
 
     float acc[4][4];
     {
