@@ -92,8 +92,12 @@ def finish_piece(backend, rank: int, initial_state, out0, qt, P_all: Sequence, H
     """What a rank does after the exchange: fold the pairs of the ranks before it into the state
     entering its piece, correct its outputs, and fold everything into the final state.
     P_all / H_all: the pairs of all ranks in rank order.  Returns (out, final_state)."""
-    S_in = backend.scan(initial_state, list(P_all[:rank]), list(H_all[:rank]))
-    out = backend.apply(S_in, qt, out0)
+    if rank == 0 and initial_state is None:
+        # the first piece of a sequence that starts from the zero state: nothing enters it
+        S_in, out = None, out0
+    else:
+        S_in = backend.scan(initial_state, list(P_all[:rank]), list(H_all[:rank]))
+        out = backend.apply(S_in, qt, out0)
     final = backend.scan(S_in, list(P_all[rank:]), list(H_all[rank:]))
     return out, final
 

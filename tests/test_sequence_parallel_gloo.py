@@ -125,3 +125,20 @@ def test_finish_piece_uses_only_earlier_ranks_for_the_entering_state():
     out, fin = finish_piece(be, 2, S0, out0, qt, P, H)
     np.testing.assert_allclose(out.numpy(), np.einsum("hvk,thk->thv", H[1][0].numpy(), qt.numpy()), atol=1e-12)
     np.testing.assert_allclose(fin.numpy(), (H[1] @ P[2] + H[2]).numpy(), atol=1e-12)
+
+
+def test_finish_piece_from_the_zero_state():
+    """initial_state = None: the first piece has nothing to correct, later pieces start from the zero state."""
+    be = OracleBackend(8, 8)
+    rng = np.random.default_rng(1)
+    H = [torch.from_numpy(rng.standard_normal((1, 2, 8, 8))) for _ in range(3)]
+    P = [torch.from_numpy(rng.standard_normal((1, 2, 8, 8))) for _ in range(3)]
+    qt = torch.from_numpy(rng.standard_normal((5, 2, 8)))
+    out0 = torch.from_numpy(rng.standard_normal((5, 2, 8)))
+    want_final = ((H[0] @ P[1] + H[1]) @ P[2] + H[2]).numpy()
+    out, fin = finish_piece(be, 0, None, out0, qt, P, H)
+    np.testing.assert_array_equal(out.numpy(), out0.numpy())
+    np.testing.assert_allclose(fin.numpy(), want_final, atol=1e-12)
+    out, fin = finish_piece(be, 1, None, out0, qt, P, H)
+    np.testing.assert_allclose(out.numpy(), out0.numpy() + np.einsum("hvk,thk->thv", H[0][0].numpy(), qt.numpy()), atol=1e-12)
+    np.testing.assert_allclose(fin.numpy(), want_final, atol=1e-12)

@@ -97,11 +97,12 @@ def test_apply_adds_state_times_carried_queries():
 
 
 @pytest.mark.parametrize("world", [2, 3, 4])
-@pytest.mark.parametrize("T,gate_mean", [(1000, 2.0), (1536, 6.0)])
-def test_emulated_ranks_match_the_oracle(world, T, gate_mean):
+@pytest.mark.parametrize("T,gate_mean,initial", [(1000, 2.0, True), (1536, 6.0, True), (700, 5.0, False), (40, 5.0, True)])
+def test_emulated_ranks_match_the_oracle(world, T, gate_mean, initial):
+    """(T = 40 with several ranks: all pieces but the first are empty.)"""
     Hqk, Hv = 2, 4
     tok = make_tokens(T, Hqk, Hv, seed=T + world, gate_mean=gate_mean)
-    init = make_state(1, Hv, seed=T)
+    init = make_state(1, Hv, seed=T) if initial else None
     spans = split_tokens(T, world)
     be = [CudaBackend() for _ in range(world)]
     parts = []
@@ -110,7 +111,7 @@ def test_emulated_ranks_match_the_oracle(world, T, gate_mean):
         parts.append(be[r].partial(d["q"], d["k"], d["v"], d["g"], d["beta"]))
     P_all = [p[3] for p in parts]  # what the all_gather would deliver
     H_all = [p[2] for p in parts]
-    S0 = torch.from_numpy(init).cuda()
+    S0 = None if init is None else torch.from_numpy(init).cuda()
     out = np.zeros((T, Hv, 128), dtype=np.float64)
     finals = []
     for r, (lo, hi) in enumerate(spans):  # phase 2 on every "rank"
