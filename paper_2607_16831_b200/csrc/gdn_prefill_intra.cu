@@ -110,9 +110,13 @@ __device__ __forceinline__ uint32_t intra_btile(int jb, int lo) {  // byte offse
 
 // FRONT: the fused entry points' q/k front end (QkFront).  q and k stay as they are in shared memory and
 // in the products; the per-token factors rq_i = scale / |q_i| and rk_j = 1 / |k_j| go into the
-// coefficients instead: A_mj gets rk_m rk_j, P_ij gets rq_i rk_j, the K-side diagonal of W and the
-// state update's e_j get rk_j, the output scaling Gamma_i gets rq_i.  The kernels after this one
-// see nothing of it.
+// coefficients instead: P_ij gets rq_i rk_j, the state update's e_j gets rk_j, the output scaling
+// Gamma_i gets rq_i.  For the triangular system, with R = diag(rk) and G = K K^T o D,
+//     A = diag(beta) R G R   and   (I + A)^-1 = R (I + diag(beta) G R^2)^-1 R^-1,
+// so the system that is solved carries only a per-COLUMN factor rk_j^2 (one scalar for the thread that
+// owns column j), and the similarity comes back at the end as a per-row factor rk_i and two rescaled
+// tables: T diag(beta) = rk_i z_ij (beta_j / rk_j), and in W = T diag(beta Gamma rk) K the column
+// factors cancel to beta_j Gamma_j.  The kernels after this one see nothing of it.
 template <bool FRONT>
 __global__ void __launch_bounds__(kIntraThreads, 4)
 gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -313,7 +317,6 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         rq[tid] = f;  // rq and rk are adjacent: thread 64 + r writes rk[r]
         __syncthreads();
         cfP[tid] *= rk[i];
-        cfA[tid] *= rk[i];
     }
     if (warp == 0 && ok) ok = mbar_wait_all(bar_mma1, 0, abort_flag);  // only this warp polls; the others park at the barrier
     ok = __syncthreads_and(ok);
@@ -405,13 +408,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                             ld16(bet + e * 64 + q4 * 16, bm);
                             // exp(gamma_m - gamma_j), m > j, as the running product of the per-token decays
                             ld16(alp + e * 64 + q4 * 16, al);
-                            float acc = FRONT ? rk[row] : 1.f;
-                            if constexpr (FRONT) {
-                                float k16[16];
-                                ld16(rk + q4 * 16, k16);
-#pragma unroll
-                                for (int x = 0; x < 16; ++x) bm[x] *= k16[x];
-                            }
+                            float acc = FRONT ? rk[row] * rk[row] : 1.f;
 #pragma unroll
                             for (int ml = 0; ml < 16; ++ml) {
                                 const bool on = q4 * 16 + ml > row;
@@ -420,7 +417,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                             }
                         } else {
                             float rf = __expf(gam[e * 64 + q4 * 16] - gi);
-                            if constexpr (FRONT) rf *= rk[row];
+                            if constexpr (FRONT) rf *= rk[row] * rk[row];
                             float cf[16];
                             ld16(cfA + e * 64 + q4 * 16, cf);
 #pragma unroll
@@ -456,6 +453,12 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         __syncthreads();  // B tiles and diagonal blocks complete; the accumulator of MMA1 is dead from here on
         tc_fence_after_sync();
         GDN_ISTAMP(2);
+        if constexpr (FRONT) {
+            // the tables of the emission below, rescaled in place (phase A is done with them; the solve's
+            // barriers come before their next use): beta_j / rk_j and Gamma_j rk_j
+            bet[tid] = bet[tid] / rk[i];
+            Gam[tid] *= rk[i];
+        }
 
         // ---- the blocked solve: z[jb][.] = columns 16 jb .. 16 jb + 15 of row i of T
         float z[4][16];
@@ -543,22 +546,18 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             //      over the B tiles, which the last step's MMAs have finished reading
             const float* bt = bet + hh * 64;
             const float* Gm = Gam + hh * 64;
+            const float rki = FRONT ? rk[i] : 1.f;
 #pragma unroll
             for (int cp = 0; cp < 4; ++cp) {  // sixteen columns at a time
                 uint32_t h1[8], l1[8], h2[8];
                 float b16[16], G16[16];
                 ld16(bt + cp * 16, b16);
                 ld16(Gm + cp * 16, G16);
-                if constexpr (FRONT) {
-                    float k16[16];
-                    ld16(rk + cp * 16, k16);
-#pragma unroll
-                    for (int x = 0; x < 16; ++x) G16[x] *= k16[x];
-                }
 #pragma unroll
                 for (int q2 = 0; q2 < 8; ++q2) {
-                    const float a0 = z[cp][q2 * 2] * b16[q2 * 2];
-                    const float a1 = z[cp][q2 * 2 + 1] * b16[q2 * 2 + 1];
+                    // (FRONT: z is a row of the similar system, the tables hold beta / rk and Gamma rk)
+                    const float a0 = (FRONT ? z[cp][q2 * 2] * rki : z[cp][q2 * 2]) * b16[q2 * 2];
+                    const float a1 = (FRONT ? z[cp][q2 * 2 + 1] * rki : z[cp][q2 * 2 + 1]) * b16[q2 * 2 + 1];
                     split_bf16x2(a0, a1, h1[q2], l1[q2]);
                     h2[q2] = pack_bf16x2(a0 * G16[q2 * 2], a1 * G16[q2 * 2 + 1]);
                 }
@@ -596,14 +595,16 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             //      operand, which MMA2 has finished reading
             uint8_t* stLo = smem + IT2 + (uint32_t)hh * 8192u;
             const float* bt = bet + hh * 64;
+            const float rki = FRONT ? rk[i] : 1.f;
 #pragma unroll
             for (int cp = 0; cp < 4; ++cp) {
                 uint32_t h1[8], l1[8];
                 float b16[16];
                 ld16(bt + cp * 16, b16);
 #pragma unroll
-                for (int q2 = 0; q2 < 8; ++q2)
-                    split_bf16x2(z[cp][q2 * 2] * b16[q2 * 2], z[cp][q2 * 2 + 1] * b16[q2 * 2 + 1], h1[q2], l1[q2]);
+                for (int q2 = 0; q2 < 8; ++q2)  // the same expressions as above: the same bits
+                    split_bf16x2((FRONT ? z[cp][q2 * 2] * rki : z[cp][q2 * 2]) * b16[q2 * 2],
+                                 (FRONT ? z[cp][q2 * 2 + 1] * rki : z[cp][q2 * 2 + 1]) * b16[q2 * 2 + 1], h1[q2], l1[q2]);
                 *reinterpret_cast<uint4*>(stLo + swz(i, 2 * cp)) = make_uint4(l1[0], l1[1], l1[2], l1[3]);
                 *reinterpret_cast<uint4*>(stLo + swz(i, 2 * cp + 1)) = make_uint4(l1[4], l1[5], l1[6], l1[7]);
             }
