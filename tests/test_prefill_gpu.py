@@ -244,3 +244,31 @@ def test_prefill_onehot_keys_associative_recall():
     rec = harness.run_prefill(dict(tokens=tok, cu_seqlens=make_cu_seqlens([T]), initial_state=None), recurrent=True)
     np.testing.assert_array_equal(rec["out"], ref_o)
     np.testing.assert_allclose(rec["final_state"], ref_s, rtol=0, atol=1e-6)
+
+
+@pytest.mark.parametrize("lengths,Hqk,Hv", [([300, 0, 65], 2, 4), ([2048], 4, 8), ([70] * 12, 1, 2)])
+def test_prefill_does_not_depend_on_what_the_workspace_and_outputs_held(lengths, Hqk, Hv):
+    """Nothing is read before it is written: the same call over a workspace and output buffers filled with
+    different garbage gives the same bits (a read of uninitialised scratch, or a result that is only
+    partly written, shows up as a difference)."""
+    import torch
+    import paper_2607_16831_b200 as gdn
+    from gdn_inputs import make_cu_seqlens, make_state, make_tokens
+    T, N = int(np.sum(lengths)), len(lengths)
+    tok = make_tokens(T, Hqk, Hv, seed=17, gate_mean=4.0)
+    d = harness.to_device(tok)
+    cu = torch.from_numpy(make_cu_seqlens(lengths)).cuda()
+    init = torch.from_numpy(make_state(N, Hv, seed=17)).cuda()
+    got = []
+    for fill in (0x00, 0xFF, 0x5A):
+        ws = harness.alloc_workspace(T, N, Hqk, Hv)
+        ws.fill_(fill)
+        out = torch.full((T, Hv, 128), 0, dtype=torch.int16, device="cuda").fill_(fill * 257 - 65536 * (fill > 127))
+        fin = torch.empty((N, Hv, 128, 128), dtype=torch.float32, device="cuda").view(torch.int32).fill_(fill * 0x01010101 - (1 << 32) * (fill > 127)).view(torch.float32)
+        gdn.gdn_prefill(d["q"], d["k"], d["v"], d["g"], d["beta"], cu, init, out.view(torch.bfloat16), fin, int(max(lengths)), ws)
+        torch.cuda.synchronize()
+        assert gdn.gdn_last_device_status(ws) == 0
+        got.append((out.cpu().numpy().copy(), fin.view(torch.int32).cpu().numpy().copy()))
+    for o, f in got[1:]:
+        np.testing.assert_array_equal(o, got[0][0])
+        np.testing.assert_array_equal(f, got[0][1])

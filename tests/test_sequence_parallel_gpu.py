@@ -122,3 +122,16 @@ def test_emulated_ranks_match_the_oracle(world, T, gate_mean, initial):
     ref_o, ref_s = oracle.prefill(tok.q, tok.k, tok.v, tok.g, tok.beta, make_cu_seqlens([T]), init)
     for fin in finals:
         harness.assert_close(out, ref_o, fin, ref_s, "sequence-parallel, %d emulated ranks" % world)
+
+
+def test_state_scan_with_no_steps_copies_the_state_every_time():
+    """steps = 0 leaves the kernel's loop empty: the result must still be written (repeated, because the
+    failure this guards against depended on what shared memory happened to hold)."""
+    S0 = torch.randn((2, 3, 128, 128), dtype=torch.float32, device="cuda")
+    for _ in range(50):
+        S_out = torch.full_like(S0, float("nan"))
+        gdn.gdn_state_scan(S0, None, None, S_out)
+        assert torch.equal(S_out, S0)
+    S_out = torch.full_like(S0, float("nan"))
+    gdn.gdn_state_scan(None, None, None, S_out)
+    assert torch.count_nonzero(S_out).item() == 0
