@@ -131,7 +131,7 @@ __device__ __forceinline__ void tc_fence_after_sync() {
 }
 
 // ---------------------------------------------------------------- TMA
-// Tiled 3-D tensor copy global -> shared (no multicast), completion on an mbarrier.
+// Tiled 3-D tensor copy global -> shared into this CTA only, completion on an mbarrier.
 __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
                                             int c2) {
     asm volatile(
