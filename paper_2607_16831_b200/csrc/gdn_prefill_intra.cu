@@ -558,6 +558,8 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     // (FRONT: z is a row of the similar system, the tables hold beta / rk and Gamma rk)
                     const float a0 = (FRONT ? z[cp][q2 * 2] * rki : z[cp][q2 * 2]) * b16[q2 * 2];
                     const float a1 = (FRONT ? z[cp][q2 * 2 + 1] * rki : z[cp][q2 * 2 + 1]) * b16[q2 * 2 + 1];
+                    z[cp][q2 * 2] = a0;  // kept for the lo parts below
+                    z[cp][q2 * 2 + 1] = a1;
                     split_bf16x2(a0, a1, h1[q2], l1[q2]);
                     h2[q2] = pack_bf16x2(a0 * G16[q2 * 2], a1 * G16[q2 * 2 + 1]);
                 }
@@ -591,20 +593,14 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         ok = __syncthreads_and(ok);
         GDN_ISTAMP(12);
         if (ok) {
-            // ---- T' lo (the bf16 remainder, recomputed from the solve's registers) -> staging over the T''
-            //      operand, which MMA2 has finished reading
+            // ---- T' lo (the bf16 remainder, split again from the values kept in registers) -> staging over
+            //      the T'' operand, which MMA2 has finished reading
             uint8_t* stLo = smem + IT2 + (uint32_t)hh * 8192u;
-            const float* bt = bet + hh * 64;
-            const float rki = FRONT ? rk[i] : 1.f;
 #pragma unroll
             for (int cp = 0; cp < 4; ++cp) {
                 uint32_t h1[8], l1[8];
-                float b16[16];
-                ld16(bt + cp * 16, b16);
 #pragma unroll
-                for (int q2 = 0; q2 < 8; ++q2)  // the same expressions as above: the same bits
-                    split_bf16x2((FRONT ? z[cp][q2 * 2] * rki : z[cp][q2 * 2]) * b16[q2 * 2],
-                                 (FRONT ? z[cp][q2 * 2 + 1] * rki : z[cp][q2 * 2 + 1]) * b16[q2 * 2 + 1], h1[q2], l1[q2]);
+                for (int q2 = 0; q2 < 8; ++q2) split_bf16x2(z[cp][q2 * 2], z[cp][q2 * 2 + 1], h1[q2], l1[q2]);
                 *reinterpret_cast<uint4*>(stLo + swz(i, 2 * cp)) = make_uint4(l1[0], l1[1], l1[2], l1[3]);
                 *reinterpret_cast<uint4*>(stLo + swz(i, 2 * cp + 1)) = make_uint4(l1[4], l1[5], l1[6], l1[7]);
             }
