@@ -108,3 +108,9 @@ def test_split_prefill_strong_decay_underflows_cleanly(gate_mean):
 def test_split_prefill_long_ragged_sequence():
     """20,001 tokens at 2/4 heads: 313 chunks in 8 runs of 40 (the last one 33 with a one-token tail)."""
     check(custom([20001], 2, 4, seed=41, gate_mean=5.0), "long ragged sequence, 8 runs")
+
+
+def test_split_prefill_quarter_million_tokens():
+    """262,161 tokens at 2/4 heads (4097 chunks, a 1 GB workspace, 8 runs of 513 chunks with a 17-token tail):
+    offsets beyond 32 bits in bytes, long chains, weak decay so that the state is carried all the way."""
+    check(custom([262144 + 17], 2, 4, seed=43, gate_mean=5.0), "quarter of a million tokens, 8 runs")
