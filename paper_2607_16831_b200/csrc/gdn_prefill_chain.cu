@@ -143,6 +143,18 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             ws + seg_block_offset(L, n, seg == 0 ? 1 : seg, h, Hv, seg == 0 ? kSegSin : (ident ? kSegP : kSegH)));
     uint16_t* out_ptr = ident ? (partial ? part.qt : reinterpret_cast<uint16_t*>(ws + L.off_qt)) : out;
 
+    // The chain warps will read their rows of the initial state (thread v: row v, four 128-byte lines) once
+    // the barriers and the tensor memory are set up; the lines are asked into L2 now, so that those
+    // loads do not pay the DRAM latency after the set-up.
+    if (warp >= kChainWarp0 && warp < kChainWarp0 + 4) {
+        if (init_ptr) {
+            const char* row = reinterpret_cast<const char*>(init_ptr + (size_t)(tid - kChainWarp0 * 32) * kD);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) prefetch_l2(row + 128 * j);
+        }
+        if ((tid & 31) == 0)
+            prefetch_l2(ws + L.off_scal + ((size_t)c_begin * Hv + h) * kScalBytes + 512);
+    }
     if (tid == 0) {
         for (int i = 0; i < B_COUNT; ++i) {
             const bool many = (i == B_DW || i == B_SHI || i == B_STM || i == B_OFREE || i == B_DL);
