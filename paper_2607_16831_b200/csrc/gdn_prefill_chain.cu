@@ -176,15 +176,18 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         return reinterpret_cast<const float*>(ws + L.off_scal + ((size_t)c * Hv + h) * kScalBytes);
     };
 #ifdef GDN_CHAIN_PROFILE
-    // SM-clock stamps of CTA 0 into the unused tail of each chunk's scalar block (4-byte slots from byte 576)
+#ifndef GDN_CHAIN_PROFILE_CTA
+#define GDN_CHAIN_PROFILE_CTA 0  // the CTA that records
+#endif
+    // SM-clock stamps of one CTA into the unused tail of each chunk's scalar block (4-byte slots from byte 576)
 // GDN_CHAIN_PROFILE is a bit mask of the stamp slots to record (every stamp costs its warp ~150 clocks)
-#define GDN_STAMP(c, slot) do { if ((((unsigned long long)(GDN_CHAIN_PROFILE) >> (slot)) & 1ull) && blockIdx.x == 0) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)(c) * Hv + h) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
+#define GDN_STAMP(c, slot) do { if ((((unsigned long long)(GDN_CHAIN_PROFILE) >> (slot)) & 1ull) && blockIdx.x == GDN_CHAIN_PROFILE_CTA) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)(c) * Hv + h) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
 #else
 #define GDN_STAMP(c, slot) do { } while (0)
 #endif
     if (tid == 0) GDN_STAMP(c_begin, 40);  // set-up done (tables read, barriers, tensor memory)
 #ifdef GDN_CHAIN_PROFILE
-    if (tid == 0 && blockIdx.x == 0)
+    if (tid == 0 && blockIdx.x == GDN_CHAIN_PROFILE_CTA)
         reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)c_begin * Hv + h) * kScalBytes + 576)[43] = t_entry;
 #endif
 
