@@ -477,9 +477,9 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         tmem_ld32(lane_addr + TM_S + b * 32, r);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<float4*>(fin_ptr + sbase + b * 32 + j) = make_float4(
-                                __uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                        for (int j = 0; j < 32; j += 8)  // 32-byte stores: every lane writes its own row
+                            st_global_v8(fin_ptr + sbase + b * 32 + j, make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]),
+                                         make_uint4(r[j + 4], r[j + 5], r[j + 6], r[j + 7]));
                         if (img) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 8)
