@@ -625,9 +625,11 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 *reinterpret_cast<uint4*>(stW + (b >> 1) * 8192 + swz(i, (b & 1) * 4 + cc)) = o;
             }
         }
+        GDN_ISTAMP(32);
         fence_proxy_async_smem();
     }
     __syncthreads();
+    GDN_ISTAMP(33);
     if (ok && i == 0 && head_ok) {
         uint8_t* wsA = ws + L.off_A + ((size_t)c * Hv + h) * kABytes;
         bulk_store(wsA + 8192, smem + IT2 + (uint32_t)hh * 8192u, 8192);  // T' lo
