@@ -108,8 +108,8 @@ static int check_prefill(const void* q, const void* k, const void* v, const floa
 }
 
 // Short-sequence dispatch of gdn_prefill.  When no sequence is longer than one chunk the chunked
-// path pays for whole 64-token chunks and three dependent launches (about 27 us even for a few
-// tokens, 13 us + 0.09 us per (sequence, head) chain beyond that), while the token-serial kernel
+// path pays for whole 64-token chunks and three dependent launches (about 22 us even for a few
+// tokens, 12 us + 0.09 us per (sequence, head) chain beyond that), while the token-serial kernel
 // costs about 0.45 us per token of the longest sequence, or 0.0052 us per token and chain once the
 // chains fill the GPU.  Both models are fits to measurements on B200 over 1..64 sequences of 4..128
 // tokens at 8 and 32 value heads; the faster one by the model is used.
@@ -121,7 +121,7 @@ static bool prefer_token_serial(int num_seqs, int Hv, int max_seqlen) {
     const double chains = (double)num_seqs * Hv;
     const double per_token = 0.0052 * chains > 0.45 ? 0.0052 * chains : 0.45;
     const double t_serial = 1.3 + 0.012 * chains + per_token * max_seqlen;
-    const double t_chunked = 13.0 + 0.092 * chains > 27.0 ? 13.0 + 0.092 * chains : 27.0;
+    const double t_chunked = 12.0 + 0.09 * chains > 22.5 ? 12.0 + 0.09 * chains : 22.5;
     return t_serial < t_chunked;
 }
 
