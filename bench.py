@@ -492,6 +492,18 @@ def run_gpu(args):
             oracle.decode(tokc.q, tokc.k, tokc.v, tokc.g, tokc.beta, cfg["state"])
             ts.append(time.perf_counter() - t0)
         med = float(np.median(ts))
+        # the timed workload's inputs, and the GPU's result on them against the oracle's (same bytes in)
+        import hashlib
+
+        hsh = hashlib.sha256()
+        for arr in (tokc.q, tokc.k, tokc.v, tokc.g, tokc.beta, cfg["state"]):
+            hsh.update(np.ascontiguousarray(arr).tobytes())
+        line["config"]["inputs"] = {"seed": rank, "sha256": hsh.hexdigest()}
+        ref_o, ref_s = oracle.decode(tokc.q, tokc.k, tokc.v, tokc.g, tokc.beta, cfg["state"])
+        chk = harness.run_decode(cfg)
+        line["parity"] = dict(harness.errors(chk["out"], ref_o, chk["state_out"], ref_s),
+                              against="the fp64 oracle on the timed workload's inputs",
+                              bounds={"out_max_abs": 2e-2, "out_rel_fro": 1e-2, "state_rel_fro": 5e-3})
         line["cpu_baseline"] = {"value": B * STATE_BYTES_PER_ITEM / med / 1e9, "unit": "GB/s",
                                 "us_per_call": med * 1e6, "cores": oracle.default_threads(), "kind": "oracle",
                                 "sample": "the full batch-64 decode workload, median of %d calls (~%.0f s of CPU work)"
