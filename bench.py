@@ -519,6 +519,10 @@ def run_gpu(args):
                 oracle.prefill(pt.q, pt.k, pt.v, pt.g, pt.beta, pc["cu_seqlens"], None)
                 reps += 1
             dt = (time.perf_counter() - t0) / reps
+            pref_o, pref_s = oracle.prefill(pt.q, pt.k, pt.v, pt.g, pt.beta, pc["cu_seqlens"], None)
+            pchk = harness.run_prefill(pc)
+            line["parity"]["prefill_long"] = dict(harness.errors(pchk["out"], pref_o, pchk["final_state"], pref_s),
+                                                  device_status=pchk["device_status"])
             line["cpu_baseline"]["prefill"] = {"tokens_per_s": 4096 / dt, "seconds_per_call": dt,
                                                "sample": "the T=4096 prefill workload (32 value heads), mean of %d calls"
                                                          % reps}
