@@ -193,6 +193,11 @@ int gdn_prefill_fused(const void* q, const void* k, const void* v, const float* 
                       const float* initial_state, void* out, float* final_state,
                       int total_tokens, int num_seqs, int max_seqlen, int Hqk, int Hv, int dk, int dv,
                       float scale, int qk_l2norm, void* workspace, size_t workspace_bytes, void* stream);
+/* gdn_decode_multi (T tokens per item, layouts as there: a, b fp32 [B,T,Hv]) with the same front end. */
+int gdn_decode_multi_fused(const void* q, const void* k, const void* v, const float* a, const float* b,
+                           const float* A_log, const float* dt_bias, const float* state_in, float* state_out,
+                           void* out, int B, int T, int Hqk, int Hv, int dk, int dv,
+                           float scale, int qk_l2norm, void* stream);
 
 /*
  * Token-serial prefill: the same inputs and outputs as gdn_prefill (no workspace),

@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL", 2: "GDN_ERR_SHAPE", 3: "GDN_ERR_
 # Every symbol include/gdn.h declares.
 EXPORTS = ("gdn_status_string", "gdn_decode", "gdn_decode_variant", "gdn_decode_num_variants",
            "gdn_prefill_workspace_bytes", "gdn_prefill", "gdn_prefill_recurrent", "gdn_prefill_static",
-           "gdn_decode_gated", "gdn_prefill_gated", "gdn_decode_fused", "gdn_prefill_fused", "gdn_decode_multi",
+           "gdn_decode_gated", "gdn_prefill_gated", "gdn_decode_fused", "gdn_prefill_fused", "gdn_decode_multi", "gdn_decode_multi_fused",
            "gdn_prefill_partial", "gdn_state_scan", "gdn_prefill_apply",
            "gdn_last_device_status")
 
@@ -70,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.gdn_decode_fused.restype = I
         L.gdn_prefill_fused.argtypes = [P] * 11 + [I] * 7 + [F, I, P, Z, P]
         L.gdn_prefill_fused.restype = I
+        L.gdn_decode_multi_fused.argtypes = [P] * 10 + [I] * 6 + [F, I, P]
+        L.gdn_decode_multi_fused.restype = I
         L.gdn_prefill_partial.argtypes = [P] * 10 + [I] * 7 + [P, Z, P]
         L.gdn_prefill_partial.restype = I
         L.gdn_state_scan.argtypes = [P, P, P, I, P, I, I, I, I, P]
@@ -228,6 +230,17 @@ def gdn_decode_fused(q, k, v, a, b, A_log, dt_bias, state_in, state_out, out, sc
                                 _ptr(state_in), _ptr(state_out), _ptr(out), B, Hqk, Hv, dk, dv, float(scale),
                                 int(bool(qk_l2norm)), _stream(stream))
     _check(rc, "gdn_decode_fused")
+
+
+def gdn_decode_multi_fused(q, k, v, a, b, A_log, dt_bias, state_in, state_out, out, scale: float = 1.0,
+                           qk_l2norm: bool = False, stream=None) -> None:
+    """gdn_decode_multi with the front end of gdn_decode_fused (a, b fp32 [B,T,Hv])."""
+    B, T, Hqk, dk = q.shape
+    _, _, Hv, dv = v.shape
+    rc = lib().gdn_decode_multi_fused(_ptr(q), _ptr(k), _ptr(v), _ptr(a), _ptr(b), _ptr(A_log), _ptr(dt_bias),
+                                      _ptr(state_in), _ptr(state_out), _ptr(out), B, T, Hqk, Hv, dk, dv, float(scale),
+                                      int(bool(qk_l2norm)), _stream(stream))
+    _check(rc, "gdn_decode_multi_fused")
 
 
 def gdn_prefill_fused(q, k, v, a, b, A_log, dt_bias, cu_seqlens, initial_state, out, final_state, max_seqlen: int,

@@ -10,8 +10,8 @@ cudaError_t decode_dispatch(const void* q, const void* k, const void* v, const f
                             const float* A_log, const float* dt_bias, const float* s_in, float* s_out, void* out,
                             int B, int Hqk, int Hv, int variant, QkFront fr, cudaStream_t st);
 cudaError_t decode_multi_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
-                                  const float* s_in, float* s_out, void* out, int B, int T, int Hqk, int Hv,
-                                  cudaStream_t st);
+                                  const float* A_log, const float* dt_bias, const float* s_in, float* s_out, void* out,
+                                  int B, int T, int Hqk, int Hv, QkFront fr, cudaStream_t st);
 cudaError_t prefill_recurrent_dispatch(const void* q, const void* k, const void* v, const float* g,
                                        const float* beta, const float* A_log, const float* dt_bias,
                                        const int32_t* cu_seqlens, const float* initial_state, void* out,
@@ -161,21 +161,31 @@ int gdn_decode_variant(const void* q, const void* k, const void* v, const float*
 
 int gdn_decode_num_variants(void) { return 12; }
 
-int gdn_decode_multi(const void* q, const void* k, const void* v, const float* g, const float* beta,
-                     const float* state_in, float* state_out, void* out, int B, int T, int Hqk, int Hv, int dk,
-                     int dv, void* stream) {
+static int decode_multi_impl(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                             const float* A_log, const float* dt_bias, const float* state_in, float* state_out,
+                             void* out, int B, int T, int Hqk, int Hv, int dk, int dv, QkFront fr, void* stream,
+                             const char* name) {
     if (B < 0 || T < 0) return GDN_ERR_SHAPE;
     if (int rc = check_heads(Hqk, Hv, dk, dv)) return rc;
     if (B == 0) return GDN_OK;
     if (!state_in || !state_out) return GDN_ERR_NULL;
     if (T > 0 && (!q || !k || !v || !g || !beta || !out)) return GDN_ERR_NULL;
+    if ((A_log == nullptr) != (dt_bias == nullptr)) return GDN_ERR_NULL;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
-        !aligned16(state_in) || !aligned16(state_out) || !aligned16(out))
+        !aligned16(state_in) || !aligned16(state_out) || !aligned16(out) ||
+        (reinterpret_cast<uintptr_t>(A_log) & 3u) || (reinterpret_cast<uintptr_t>(dt_bias) & 3u))
         return GDN_ERR_ALIGN;
     if ((long long)B * Hv * 32 > 0x7fffffffLL || (long long)B * T > 0x7fffffffLL) return GDN_ERR_SHAPE;
     if (!device_supported()) return GDN_ERR_UNSUPPORTED;
-    return cuda_status(decode_multi_dispatch(q, k, v, g, beta, state_in, state_out, out, B, T, Hqk, Hv,
-                                             (cudaStream_t)stream), "gdn_decode_multi");
+    return cuda_status(decode_multi_dispatch(q, k, v, g, beta, A_log, dt_bias, state_in, state_out, out, B, T, Hqk, Hv,
+                                             fr, (cudaStream_t)stream), name);
+}
+
+int gdn_decode_multi(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                     const float* state_in, float* state_out, void* out, int B, int T, int Hqk, int Hv, int dk,
+                     int dv, void* stream) {
+    return decode_multi_impl(q, k, v, g, beta, nullptr, nullptr, state_in, state_out, out, B, T, Hqk, Hv, dk, dv,
+                             QkFront{1.f, 0}, stream, "gdn_decode_multi");
 }
 
 size_t gdn_prefill_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int Hv, int dk, int dv) {
@@ -226,6 +236,15 @@ int gdn_decode_fused(const void* q, const void* k, const void* v, const float* a
     if (B > 0 && ((A_log == nullptr) != (dt_bias == nullptr))) return GDN_ERR_NULL;
     return decode_impl(q, k, v, a, b, A_log, dt_bias, A_log != nullptr, state_in, state_out, out, B, Hqk, Hv, dk, dv,
                        -1, QkFront{scale, qk_l2norm != 0}, stream);
+}
+
+int gdn_decode_multi_fused(const void* q, const void* k, const void* v, const float* a, const float* b,
+                           const float* A_log, const float* dt_bias, const float* state_in, float* state_out,
+                           void* out, int B, int T, int Hqk, int Hv, int dk, int dv, float scale, int qk_l2norm,
+                           void* stream) {
+    if (!front_ok(scale)) return GDN_ERR_SHAPE;
+    return decode_multi_impl(q, k, v, a, b, A_log, dt_bias, state_in, state_out, out, B, T, Hqk, Hv, dk, dv,
+                             QkFront{scale, qk_l2norm != 0}, stream, "gdn_decode_multi_fused");
 }
 
 // gdn_prefill_gated and gdn_prefill_fused: raw gates when A_log / dt_bias are given, and the q/k front end

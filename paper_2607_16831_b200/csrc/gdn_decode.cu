@@ -195,12 +195,14 @@ cudaError_t decode_dispatch(const void* q, const void* k, const void* v, const f
 // Multi-token decode: T tokens per batch item (speculative / chunked decode), applied in order to
 // state rows that stay in registers, so the state is still read once and written once.
 // Layouts: q,k [B,T,Hqk,128], v,out [B,T,Hv,128], g,beta [B,T,Hv].
-template <int NB, int WARPS>
+// FRONT: raw gate inputs when A_log is given, and the q/k front end `fr` (the fused entry point).
+template <int NB, int WARPS, bool FRONT>
 __global__ void __launch_bounds__(WARPS * 32)
 gdn_decode_multi_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
                         const uint16_t* __restrict__ v, const float* __restrict__ g,
-                        const float* __restrict__ beta, const float* s_in, float* s_out,
-                        uint16_t* __restrict__ out, int T, int Hqk, int Hv, int split) {
+                        const float* __restrict__ beta, const float* __restrict__ A_log,
+                        const float* __restrict__ dt_bias, const float* s_in, float* s_out,
+                        uint16_t* __restrict__ out, int T, int Hqk, int Hv, int split, QkFront fr) {
     pdl_wait();
     pdl_launch_dependents();
     const int cta = blockIdx.x;
@@ -234,13 +236,34 @@ gdn_decode_multi_kernel(const uint16_t* __restrict__ q, const uint16_t* __restri
             unpack_bf16x2(qw.x, qf[4 * j + 0], qf[4 * j + 1]);
             unpack_bf16x2(qw.y, qf[4 * j + 2], qf[4 * j + 3]);
         }
-        const float alpha = __expf(__ldg(g + tok * Hv + h));
-        const float bt = __ldg(beta + tok * Hv + h);
+        float gl = __ldg(g + tok * Hv + h), bt = __ldg(beta + tok * Hv + h);
+        if (FRONT && A_log) raw_gates(gl, bt, __ldg(A_log + h), __ldg(dt_bias + h), gl, bt);
+        const float alpha = __expf(gl);
         float qk = 0.f;
 #pragma unroll
         for (int j = 0; j < 16; ++j) qk = fmaf(qf[j], kf[j], qk);
 #pragma unroll
         for (int m = 1; m < 8; m <<= 1) qk += __shfl_xor_sync(0xffffffffu, qk, m);
+        float rk = 1.f, rq = 1.f;
+        if constexpr (FRONT) {
+            rq = fr.scale;
+            if (fr.l2norm) {
+                float kk = 0.f, qq = 0.f;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    kk = fmaf(kf[j], kf[j], kk);
+                    qq = fmaf(qf[j], qf[j], qq);
+                }
+#pragma unroll
+                for (int m = 1; m < 8; m <<= 1) {
+                    kk += __shfl_xor_sync(0xffffffffu, kk, m);
+                    qq += __shfl_xor_sync(0xffffffffu, qq, m);
+                }
+                rk = rsqrtf(kk + kNormEps);
+                rq *= rsqrtf(qq + kNormEps);
+            }
+            qk *= rk * rq;
+        }
         const uint16_t* v_h = v + (tok * Hv + h) * kD;
         uint16_t* o_h = out + (tok * Hv + h) * kD;
 #pragma unroll
@@ -262,15 +285,16 @@ gdn_decode_multi_kernel(const uint16_t* __restrict__ q, const uint16_t* __restri
                 a += __shfl_xor_sync(0xffffffffu, a, m);
                 p += __shfl_xor_sync(0xffffffffu, p, m);
             }
-            const float delta = bt * (bf16_bits_to_float(__ldg(v_h + row0 + i * 4 + sub)) - alpha * a);
+            const float delta = bt * (bf16_bits_to_float(__ldg(v_h + row0 + i * 4 + sub)) - alpha * (FRONT ? a * rk : a));
+            const float dk = FRONT ? delta * rk : delta;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                s[i][j].x = fmaf(alpha, s[i][j].x, delta * kf[4 * j + 0]);
-                s[i][j].y = fmaf(alpha, s[i][j].y, delta * kf[4 * j + 1]);
-                s[i][j].z = fmaf(alpha, s[i][j].z, delta * kf[4 * j + 2]);
-                s[i][j].w = fmaf(alpha, s[i][j].w, delta * kf[4 * j + 3]);
+                s[i][j].x = fmaf(alpha, s[i][j].x, dk * kf[4 * j + 0]);
+                s[i][j].y = fmaf(alpha, s[i][j].y, dk * kf[4 * j + 1]);
+                s[i][j].z = fmaf(alpha, s[i][j].z, dk * kf[4 * j + 2]);
+                s[i][j].w = fmaf(alpha, s[i][j].w, dk * kf[4 * j + 3]);
             }
-            if (c == 0) o_h[row0 + i * 4 + sub] = float_to_bf16_bits(fmaf(delta, qk, alpha * p));
+            if (c == 0) o_h[row0 + i * 4 + sub] = float_to_bf16_bits(fmaf(delta, qk, alpha * (FRONT ? p * rq : p)));
         }
     }
 #pragma unroll
@@ -281,29 +305,30 @@ gdn_decode_multi_kernel(const uint16_t* __restrict__ q, const uint16_t* __restri
     }
 }
 
+template <int NB, int WARPS>
+static cudaError_t launch_multi(const void* q, const void* k, const void* v, const float* g, const float* beta,
+                                const float* A_log, const float* dt_bias, const float* s_in, float* s_out, void* out,
+                                int B, int T, int Hqk, int Hv, QkFront fr, cudaStream_t st) {
+    constexpr int split = kD / (WARPS * 4 * NB);
+    const dim3 grid((unsigned)((long long)B * Hv * split));
+    if (A_log || fr.active())
+        return launch_pdl(gdn_decode_multi_kernel<NB, WARPS, true>, grid, dim3(WARPS * 32), 0, st, (const uint16_t*)q,
+                          (const uint16_t*)k, (const uint16_t*)v, g, beta, A_log, dt_bias, s_in, s_out, (uint16_t*)out,
+                          T, Hqk, Hv, split, fr);
+    return launch_pdl(gdn_decode_multi_kernel<NB, WARPS, false>, grid, dim3(WARPS * 32), 0, st, (const uint16_t*)q,
+                      (const uint16_t*)k, (const uint16_t*)v, g, beta, A_log, dt_bias, s_in, s_out, (uint16_t*)out, T,
+                      Hqk, Hv, split, fr);
+}
+
 cudaError_t decode_multi_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
-                                  const float* s_in, float* s_out, void* out, int B, int T, int Hqk, int Hv,
-                                  cudaStream_t st) {
-    if (B <= 2) {
-        constexpr int NB = 1, WARPS = 1, split = kD / (WARPS * 4 * NB);
-        return launch_pdl(gdn_decode_multi_kernel<NB, WARPS>, dim3((unsigned)((long long)B * Hv * split)),
-                          dim3(WARPS * 32), 0, st, (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta,
-                          s_in, s_out, (uint16_t*)out, T, Hqk, Hv, split);
-    } else if (B >= 32) {
-        // Bandwidth regime: with T tokens per state row the kernel is co-bound by instruction issue
-        // (every token costs a warp ~90 instructions that do not depend on how many rows it owns), so
-        // sixteen rows per warp beat eight (B = 64, T = 4: 50.7 vs 58.1 us; 32 rows run out of registers).
-        constexpr int NB = 4, WARPS = 2, split = kD / (WARPS * 4 * NB);
-        return launch_pdl(gdn_decode_multi_kernel<NB, WARPS>, dim3((unsigned)((long long)B * Hv * split)),
-                          dim3(WARPS * 32), 0, st, (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta,
-                          s_in, s_out, (uint16_t*)out, T, Hqk, Hv, split);
-    } else {
-        constexpr int NB = 2, WARPS = 4, split = kD / (WARPS * 4 * NB);
-        return launch_pdl(gdn_decode_multi_kernel<NB, WARPS>, dim3((unsigned)((long long)B * Hv * split)),
-                          dim3(WARPS * 32), 0, st, (const uint16_t*)q, (const uint16_t*)k, (const uint16_t*)v, g, beta,
-                          s_in, s_out, (uint16_t*)out, T, Hqk, Hv, split);
-    }
-    return cudaGetLastError();
+                                  const float* A_log, const float* dt_bias, const float* s_in, float* s_out, void* out,
+                                  int B, int T, int Hqk, int Hv, QkFront fr, cudaStream_t st) {
+    if (B <= 2) return launch_multi<1, 1>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, T, Hqk, Hv, fr, st);
+    // Bandwidth regime: with T tokens per state row the kernel is co-bound by instruction issue
+    // (every token costs a warp ~90 instructions that do not depend on how many rows it owns), so
+    // sixteen rows per warp beat eight (B = 64, T = 4: 50.7 vs 58.1 us; 32 rows run out of registers).
+    if (B >= 32) return launch_multi<4, 2>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, T, Hqk, Hv, fr, st);
+    return launch_multi<2, 4>(q, k, v, g, beta, A_log, dt_bias, s_in, s_out, out, B, T, Hqk, Hv, fr, st);
 }
 
 }  // namespace gdn

@@ -68,6 +68,13 @@ def test_host_side_argument_checks(gdn):
     assert L.gdn_decode_fused(fake, fake, fake, fake, fake, None, None, fake, fake, fake, 2, 16, 32, 128, 128,
                               float("inf"), 1, None) == 2
     assert L.gdn_decode_fused(fake, fake, fake, fake, fake, None, None, fake, fake, fake, 0, 16, 32, 128, 128, 1.0, 1, None) == 0
+    assert L.gdn_decode_multi_fused(fake, fake, fake, fake, fake, fake, None, fake, fake, fake, 2, 3, 16, 32, 128, 128,
+                                    1.0, 1, None) == 1
+    assert L.gdn_decode_multi_fused(fake, fake, fake, fake, fake, None, None, fake, fake, fake, 2, -1, 16, 32, 128, 128,
+                                    1.0, 1, None) == 2
+    assert L.gdn_decode_multi_fused(fake, fake, fake, fake, fake, None, None, fake, fake, fake, 2, 3, 16, 32, 128, 128,
+                                    float("inf"), 0, None) == 2
+    assert L.gdn_decode_multi(fake, fake, odd, fake, fake, fake, fake, fake, 2, 3, 16, 32, 128, 128, None) == 5
     fa = [fake] * 11
     assert L.gdn_prefill_fused(*fa, 100, 2, 60, 16, 32, 128, 128, float("nan"), 0, fake, 1 << 30, None) == 2
     a = list(fa); a[5] = None   # A_log without dt_bias

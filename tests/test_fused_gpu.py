@@ -77,6 +77,35 @@ def test_decode_fused_matches_oracle(B, raw, scale, l2norm):
     assert e["state_rel_fro"] < 2e-6
 
 
+@pytest.mark.parametrize("B,T", [(1, 3), (6, 4), (40, 2)])
+@pytest.mark.parametrize("raw,scale,l2norm", [(True, 0.5, True), (False, 0.25, False)])
+def test_decode_multi_fused_matches_oracle(B, T, raw, scale, l2norm):
+    """T tokens per item in one pass over the state, with the front end: the oracle's fused prefill over B
+    sequences of length T from the same states."""
+    import torch
+    import paper_2607_16831_b200 as gdn
+    Hqk, Hv = 4, 8
+    tok = make_tokens(B * T, Hqk, Hv, seed=300 + B + T, gate_mean=3.0)
+    qb, kb = unnormalised(tok, B + T) if l2norm else (tok.q, tok.k)
+    if raw:
+        a, b, A_log, dt_bias = make_raw_gates(B * T, Hv, seed=B + T)
+    else:
+        a, b, A_log, dt_bias = tok.g, tok.beta, None, None
+    st = make_state(B, Hv, seed=300 + B)
+    shp = lambda bits, H: harness.bf16_to_device(bits).view(B, T, H, 128)
+    s_in = _dev(st)
+    s_out = torch.full_like(s_in, float("nan"))
+    out = torch.full((B, T, Hv, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    gdn.gdn_decode_multi_fused(shp(qb, Hqk), shp(kb, Hqk), shp(tok.v, Hv), _dev(a).view(B, T, Hv), _dev(b).view(B, T, Hv),
+                               _dev(A_log), _dev(dt_bias), s_in, s_out, out, scale=scale, qk_l2norm=l2norm)
+    torch.cuda.synchronize()
+    ref_o, ref_s = oracle.prefill_fused(qb, kb, tok.v, a, b, A_log, dt_bias, make_cu_seqlens([T] * B), st, scale=scale,
+                                        qk_l2norm=l2norm)
+    e = harness.assert_close(harness.bf16_to_numpy(out).reshape(B * T, Hv, 128), ref_o,
+                             s_out.cpu().numpy().astype(np.float64), ref_s, "decode multi fused B=%d T=%d" % (B, T))
+    assert e["state_rel_fro"] < 5e-6
+
+
 CASES = [
     ([64], 1, 1, "one chunk"),
     ([200, 1, 77], 2, 4, "ragged chunks, three sequences"),
