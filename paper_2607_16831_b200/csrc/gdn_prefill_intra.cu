@@ -348,6 +348,19 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 uint32_t r[16];
                 tmem_ld16(lane_addr + ITM_D1 + q4 * 16, r);
                 tmem_ld_wait();
+                // A side: the two half warps own different diagonal blocks (16 j_own and the one right of it).
+                // Both are handled in the same iteration, the first of the warp's two, so that the
+                // per-element code runs once for all 32 lanes instead of once per half warp: the upper half
+                // takes its sixteen columns from a second load.
+                const int wbA = (row >> 5) * 2;
+                uint32_t xd[16];
+                if (tid >= 64 && q4 == wbA) {
+                    uint32_t r2[16];
+                    tmem_ld16(lane_addr + ITM_D1 + (q4 + 1) * 16, r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int ml = 0; ml < 16; ++ml) xd[ml] = (row & 16) ? r2[ml] : r[ml];
+                }
 #pragma unroll 1
                 for (int e = 0; e < 2; ++e) {
                     const float* gm = gam + e * 64 + q4 * 16;
@@ -401,19 +414,20 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                             st_swizzled_pair(wsP, (uint32_t)row, (uint32_t)q4, make_uint4(pk[0], pk[1], pk[2], pk[3]),
                                              make_uint4(pk[4], pk[5], pk[6], pk[7]));
                         }
-                    } else if (q4 >= jb_own) {
+                    } else if (q4 == wbA || q4 > jb_own) {
                         float a[16];
-                        if (q4 == jb_own) {
+                        const bool diag = q4 == wbA;
+                        if (diag) {
                             float bm[16], al[16];
-                            ld16(bet + e * 64 + q4 * 16, bm);
+                            ld16(bet + e * 64 + jb_own * 16, bm);
                             // exp(gamma_m - gamma_j), m > j, as the running product of the per-token decays
-                            ld16(alp + e * 64 + q4 * 16, al);
+                            ld16(alp + e * 64 + jb_own * 16, al);
                             float acc = FRONT ? rk[row] * rk[row] : 1.f;
 #pragma unroll
                             for (int ml = 0; ml < 16; ++ml) {
-                                const bool on = q4 * 16 + ml > row;
+                                const bool on = jb_own * 16 + ml > row;
                                 acc = on ? acc * al[ml] : acc;
-                                a[ml] = on ? bm[ml] * acc * __uint_as_float(r[ml]) : 0.f;
+                                a[ml] = on ? bm[ml] * acc * __uint_as_float(xd[ml]) : 0.f;
                             }
                         } else {
                             float rf = __expf(gam[e * 64 + q4 * 16] - gi);
@@ -423,7 +437,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
                             for (int ml = 0; ml < 16; ++ml) a[ml] = (rf * cf[ml]) * __uint_as_float(r[ml]);
                         }
-                        if (q4 == jb_own) {
+                        if (diag) {
                             // stored by row m: the solve reads, for one m, the run of columns j < m as float4s
                             float* dg = reinterpret_cast<float*>(smem + IDG) + (e * 4 + jb_own) * 256 + (row & 15);
 #pragma unroll
