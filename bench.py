@@ -88,6 +88,13 @@ class ClockSampler:
         if self._nv is not None:
             self._thread = threading.Thread(target=self._run, daemon=True)
             self._thread.start()
+            # the first queries of a process can take tens of milliseconds inside the driver: let them happen
+            # before the timed region starts, then drop what they returned
+            t0 = time.perf_counter()
+            while len(self.samples) < 3 and time.perf_counter() - t0 < 0.25:
+                time.sleep(0.002)
+            self.samples.clear()
+            self.reasons.clear()
         return self
 
     def __exit__(self, *a):
