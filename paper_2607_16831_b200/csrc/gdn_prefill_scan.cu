@@ -20,8 +20,7 @@
 namespace gdn {
 using namespace sm100;
 
-constexpr int kCombineRows = 16;
-constexpr uint32_t CB_XT = 0;        // X transposed: xt[k][row] fp32                 8 KB
+constexpr uint32_t CB_XT = 0;        // X transposed: xt[k][row] fp32                 up to 8 KB
 constexpr uint32_t CB_BAR = 8192;    // two mbarriers, abort flag
 constexpr uint32_t CB_P = 8192 + 128;  // one or two buffers of P, fp32 [128][128]   64 KB each
 constexpr uint32_t kPBlock = (uint32_t)kSegBlockBytes;
@@ -44,13 +43,17 @@ struct ScanArgs {
     int* status;            // device status word
 };
 
-// grid (sequences x value heads, 128 / 16 row blocks).  `nbuf` = 2 fetches the next step's P while
-// this step's product is computed.
+// grid (sequences x value heads, 128 / (4 RW) row blocks): a CTA owns 4 RW rows of the state, a thread RW rows
+// x 4 columns.  RW = 2 doubles the CTAs per (sequence, head) when there are few of those (the steps are
+// serial, so this is the only parallelism there is).  `nbuf` = 2 fetches the next step's P while this step's
+// product is computed.
+template <int RW>
 __global__ void __launch_bounds__(128)
 gdn_prefill_combine_kernel(ScanArgs A, int Hv, int nbuf) {
+    constexpr int kCombineRows = 4 * RW;
     const int n = blockIdx.x / Hv, h = blockIdx.x % Hv;
     const int row0 = blockIdx.y * kCombineRows;
-    const int tid = threadIdx.x, ty = tid >> 5, tx = tid & 31;  // thread tile: rows 4 ty.., columns 4 tx..
+    const int tid = threadIdx.x, ty = tid >> 5, tx = tid & 31;  // thread tile: rows RW ty.., columns 4 tx..
     const int nch = A.chunk_off ? A.chunk_off[n + 1] - A.chunk_off[n] : 1;
     if (nch <= 0) return;  // empty sequence: the chain kernel passed the state through
     const long long unit = (long long)n * A.sn + (long long)h * A.sh;
@@ -85,13 +88,13 @@ gdn_prefill_combine_kernel(ScanArgs A, int Hv, int nbuf) {
     }
     __syncthreads();  // the barriers and the abort flag are set before anybody reads them (the loop below may run zero times)
 
-    float acc[4][4];
+    float acc[RW][4];
     {
         const float* x0 = A.x0 ? A.x0 + (long long)n * A.x_sn + (long long)h * A.x_sh : nullptr;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < RW; ++i) {
             float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (x0) x = *reinterpret_cast<const float4*>(x0 + (size_t)(row0 + ty * 4 + i) * kD + tx * 4);
+            if (x0) x = *reinterpret_cast<const float4*>(x0 + (size_t)(row0 + ty * RW + i) * kD + tx * 4);
             acc[i][0] = x.x; acc[i][1] = x.y; acc[i][2] = x.z; acc[i][3] = x.w;
         }
     }
@@ -102,8 +105,8 @@ gdn_prefill_combine_kernel(ScanArgs A, int Hv, int nbuf) {
             float* sin = A.sin + (long long)(s - 1) * A.ss + unit;
             uint8_t* img = A.img + ((long long)(s - 1) * A.ss + unit) * 4;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int r = row0 + ty * 4 + i;
+            for (int i = 0; i < RW; ++i) {
+                const int r = row0 + ty * RW + i;
                 *reinterpret_cast<float4*>(sin + (size_t)r * kD + tx * 4) =
                     make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
                 *reinterpret_cast<uint2*>(img + (tx >> 4) * 16384 + swz((uint32_t)r, (uint32_t)((tx >> 1) & 7)) + (tx & 1) * 8) =
@@ -111,17 +114,21 @@ gdn_prefill_combine_kernel(ScanArgs A, int Hv, int nbuf) {
             }
         }
         const float* H = A.H + (long long)(s - 1) * A.ss + unit;
-        float4 hrow[4];
+        float4 hrow[RW];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) hrow[i] = *reinterpret_cast<const float4*>(H + (size_t)(row0 + ty * 4 + i) * kD + tx * 4);
+        for (int i = 0; i < RW; ++i) hrow[i] = *reinterpret_cast<const float4*>(H + (size_t)(row0 + ty * RW + i) * kD + tx * 4);
         __syncthreads();  // the previous step's reads of xt and of the other P buffer are done
         if (tid == 0 && nbuf == 2 && run_chunks(s + 1) > 0) fetch_P(s + 1);
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-            *reinterpret_cast<float4*>(&xt[tx * 4 + j][ty * 4]) = make_float4(acc[0][j], acc[1][j], acc[2][j], acc[3][j]);
+        for (int j = 0; j < 4; ++j) {
+            if constexpr (RW == 4)
+                *reinterpret_cast<float4*>(&xt[tx * 4 + j][ty * 4]) = make_float4(acc[0][j], acc[1][j], acc[2][j], acc[3][j]);
+            else
+                *reinterpret_cast<float2*>(&xt[tx * 4 + j][ty * 2]) = make_float2(acc[0][j], acc[1][j]);
+        }
         __syncthreads();
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < RW; ++i) {
             acc[i][0] = hrow[i].x; acc[i][1] = hrow[i].y; acc[i][2] = hrow[i].z; acc[i][3] = hrow[i].w;
         }
         const int b = (s - 1) % nbuf;
@@ -130,10 +137,16 @@ gdn_prefill_combine_kernel(ScanArgs A, int Hv, int nbuf) {
 #pragma unroll 8
         for (int k = 0; k < kD; ++k) {
             const float4 p = *reinterpret_cast<const float4*>(P + k * kD + tx * 4);
-            const float4 x = *reinterpret_cast<const float4*>(&xt[k][ty * 4]);
-            const float xr[4] = {x.x, x.y, x.z, x.w};
+            float xr[RW];
+            if constexpr (RW == 4) {
+                const float4 x = *reinterpret_cast<const float4*>(&xt[k][ty * 4]);
+                xr[0] = x.x; xr[1] = x.y; xr[2] = x.z; xr[3] = x.w;
+            } else {
+                const float2 x = *reinterpret_cast<const float2*>(&xt[k][ty * 2]);
+                xr[0] = x.x; xr[1] = x.y;
+            }
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < RW; ++i) {
                 acc[i][0] = fmaf(xr[i], p.x, acc[i][0]);
                 acc[i][1] = fmaf(xr[i], p.y, acc[i][1]);
                 acc[i][2] = fmaf(xr[i], p.z, acc[i][2]);
@@ -152,8 +165,8 @@ gdn_prefill_combine_kernel(ScanArgs A, int Hv, int nbuf) {
     if (A.fin) {
         float* fin = A.fin + ((size_t)n * Hv + h) * kD * kD;
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-            *reinterpret_cast<float4*>(fin + (size_t)(row0 + ty * 4 + i) * kD + tx * 4) =
+        for (int i = 0; i < RW; ++i)
+            *reinterpret_cast<float4*>(fin + (size_t)(row0 + ty * RW + i) * kD + tx * 4) =
                 make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
     }
 }
@@ -287,12 +300,28 @@ gdn_prefill_fixup_kernel(const __grid_constant__ CUtensorMap map_out, const __gr
     }
 }
 
+// Launch shape of the combine kernel: 16-row CTAs (eight per sequence and head), or 8-row CTAs when even
+// twice as many still leave SMs idle; two P buffers (a whole SM per CTA) when there are several steps and the
+// grid is small enough for it.
+static void launch_combine(const ScanArgs& A, int num_seqs, int Hv, bool several_steps, cudaStream_t st) {
+    const long long units = (long long)num_seqs * Hv;
+    if (units * 16 <= kAssumedSMs) {
+        const int nbuf = several_steps ? 2 : 1;
+        gdn_prefill_combine_kernel<2><<<dim3((unsigned)units, 16), 128, combine_smem(nbuf), st>>>(A, Hv, nbuf);
+    } else {
+        const int nbuf = (several_steps && units * 8 <= kAssumedSMs) ? 2 : 1;
+        gdn_prefill_combine_kernel<4><<<dim3((unsigned)units, 8), 128, combine_smem(nbuf), st>>>(A, Hv, nbuf);
+    }
+}
+
 static cudaError_t scan_attrs() {
     static bool attr_done[64];
     return set_attrs_once(attr_done, [] {
         cudaError_t e = cudaFuncSetAttribute(gdn_prefill_fixup_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFixSmem);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(gdn_prefill_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, combine_smem(2));
+            e = cudaFuncSetAttribute(gdn_prefill_combine_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, combine_smem(2));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(gdn_prefill_combine_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, combine_smem(2));
         return e;
     });
 }
@@ -302,9 +331,6 @@ cudaError_t launch_prefill_scan(const CUtensorMap& mout, const CUtensorMap& mqt,
                                 cudaStream_t st) {
     if (segs <= 1) return cudaSuccess;
     if (cudaError_t e = scan_attrs()) return e;
-    const dim3 cgrid((unsigned)(num_seqs * Hv), kD / kCombineRows);
-    // two P buffers need a whole SM per CTA: worth it when there are several steps and the grid is small
-    const int nbuf = (segs > 2 && (long long)cgrid.x * cgrid.y <= kAssumedSMs) ? 2 : 1;
     ScanArgs A;
     const long long blk = (long long)(kSegBlockBytes / sizeof(float));
     float* seg0 = reinterpret_cast<float*>(ws + L.off_seg);
@@ -325,13 +351,13 @@ cudaError_t launch_prefill_scan(const CUtensorMap& mout, const CUtensorMap& mqt,
     A.status = reinterpret_cast<int*>(ws);
     // states entering runs 2.. come out of the combine; with two runs the fix-up only needs run 0's
     // final state, so the combine (then only the final state) goes last
-    if (segs > 2) gdn_prefill_combine_kernel<<<cgrid, 128, combine_smem(nbuf), st>>>(A, Hv, nbuf);
+    if (segs > 2) launch_combine(A, num_seqs, Hv, true, st);
     const int max_chunks = (max_seqlen + kChunk - 1) / kChunk;
     const int seg_chunks = (max_chunks + segs - 1) / segs;
     const dim3 fgrid((unsigned)((seg_chunks * kChunk + kFixTokens - 1) / kFixTokens), (unsigned)Hv,
                      (unsigned)(num_seqs * (segs - 1)));
     gdn_prefill_fixup_kernel<<<fgrid, 128, kFixSmem, st>>>(mout, mqt, (uint16_t*)out, ws, L, Hv, segs, nullptr, nullptr);
-    if (segs == 2 && final_state) gdn_prefill_combine_kernel<<<cgrid, 128, combine_smem(nbuf), st>>>(A, Hv, nbuf);
+    if (segs == 2 && final_state) launch_combine(A, num_seqs, Hv, false, st);
     return cudaGetLastError();
 }
 
@@ -356,8 +382,6 @@ __global__ void __launch_bounds__(128) gdn_state_image_kernel(const float* __res
 cudaError_t launch_state_scan(const float* S0, const float* P, const float* H, int steps, float* S_out, int num_seqs,
                               int Hv, cudaStream_t st) {
     if (cudaError_t e = scan_attrs()) return e;
-    const dim3 cgrid((unsigned)(num_seqs * Hv), kD / kCombineRows);
-    const int nbuf = (steps > 1 && (long long)cgrid.x * cgrid.y <= kAssumedSMs) ? 2 : 1;
     ScanArgs A;
     const long long blk = (long long)kD * kD;
     A.x0 = S0;
@@ -375,7 +399,7 @@ cudaError_t launch_state_scan(const float* S0, const float* P, const float* H, i
     A.chunk_off = nullptr;
     A.segs = 0;
     A.status = nullptr;
-    gdn_prefill_combine_kernel<<<cgrid, 128, combine_smem(nbuf), st>>>(A, Hv, nbuf);
+    launch_combine(A, num_seqs, Hv, steps > 1, st);
     return cudaGetLastError();
 }
 
