@@ -165,3 +165,33 @@ def test_decode_from_host_buffers_in_slices(B, slices, streams):
     ref_o2, ref_s2 = oracle.decode(*harness.token_arrays(tok), ref_s.astype(np.float32))
     harness.assert_close(harness.bf16_to_numpy(h_out.view(torch.bfloat16)), ref_o2,
                          h_state_out.numpy().astype(np.float64), ref_s2, "host decode, second step")
+
+
+@pytest.mark.parametrize("B,slices,streams", [(12, 4, 2), (7, 8, 3), (3, 1, 1)])
+def test_host_decode_steps_enqueued_back_to_back(B, slices, streams):
+    """Five steps with different inputs enqueued without synchronising in between (they overlap on the device:
+    one step's copies back run while the next step's inputs come in), each with its own host output buffers;
+    every step must match the oracle on its own inputs: the reuse of the device buffers is ordered."""
+    import torch
+    from gdn_inputs import config
+    from paper_2607_16831_b200.host_pipeline import HostDecode
+
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    steps = []
+    for s in range(5):
+        cfg = config("decode_sweep", B=B, seed=40 + s)
+        tok, st = cfg["tokens"], cfg["state"]
+        steps.append(dict(tok=tok, st=st,
+                          h=[pin(tok.q.view(np.int16)), pin(tok.k.view(np.int16)), pin(tok.v.view(np.int16)), pin(tok.g),
+                             pin(tok.beta)],
+                          h_state=pin(st),
+                          h_out=torch.full((B, tok.Hv, 128), -1, dtype=torch.int16).pin_memory(),
+                          h_state_out=torch.full((B, tok.Hv, 128, 128), float("nan"), dtype=torch.float32).pin_memory()))
+    pipe = HostDecode(B, steps[0]["tok"].Hqk, steps[0]["tok"].Hv, slices=slices, streams=streams)
+    for x in steps:
+        pipe.step(*x["h"], x["h_state"], x["h_state_out"], x["h_out"])
+    torch.cuda.current_stream().synchronize()  # the caller's stream waits for every step's last copy
+    for s, x in enumerate(steps):
+        ref_o, ref_s = oracle.decode(*harness.token_arrays(x["tok"]), x["st"])
+        harness.assert_close(harness.bf16_to_numpy(x["h_out"].view(torch.bfloat16)), ref_o,
+                             x["h_state_out"].numpy().astype(np.float64), ref_s, "host decode, step %d of 5" % s)
