@@ -479,6 +479,21 @@ def run_gpu(args):
         pre.append(dict(bench_prefill("short", peaks, reps, lengths=[8] * 64, Hqk=4, Hv=8,
                                       env={"GDN_PREFILL_SHORT_FALLBACK": "0"}),
                         variant="4/8 heads, 64 sequences of 8 tokens, chunked kernels forced"))
+        # many short sequences at 4 key / 8 value heads (the shape of the paper's contest workloads): which path the
+        # library takes and what it costs, against the other path forced
+        if not args.quick:
+            sweep_short = []
+            for nseq, ln in ((16, 16), (64, 32), (256, 8), (256, 48), (64, 128), (256, 256)):
+                auto = bench_prefill("short", peaks, 8, lengths=[ln] * nseq, Hqk=4, Hv=8)["us"]
+                chunked = bench_prefill("short", peaks, 8, lengths=[ln] * nseq, Hqk=4, Hv=8,
+                                        env={"GDN_PREFILL_SHORT_FALLBACK": "0"})["us"]
+                sweep_short.append({"num_seqs": nseq, "len": ln, "us": auto, "us_chunked_forced": chunked,
+                                    "tokens_per_s": nseq * ln / (auto * 1e-6)})
+            short_sweep_result = {"heads": "4/8", "note": "cold single calls; equal `us` means the chunked path was "
+                                                         "chosen by the dispatch (always so above 64 tokens)",
+                                  "points": sweep_short}
+        else:
+            short_sweep_result = None
         # µs per chunk step of the serial chain: one sequence of 4096 tokens against two of 2048 (the same
         # intra-chunk work, 32 more dependent steps), sequence split switched off
         off = {"GDN_PREFILL_MAX_SEGMENTS": "1"}
@@ -488,6 +503,8 @@ def run_gpu(args):
                                          "bytes_per_token": PREFILL_BYTES_PER_TOKEN,
                                          "flops_per_token": PREFILL_FLOPS_PER_TOKEN},
                            "chain_us_per_chunk_step": (t64 - t32) / 32.0, "runs": pre}
+        if short_sweep_result is not None:
+            line["prefill"]["short_sequence_sweep"] = short_sweep_result
         # ---- CPU oracle on this machine's host cores (reported baseline, not the target)
         import oracle
 
