@@ -22,9 +22,10 @@
  *     required for every tensor pointer.
  *   - Only dk = dv = 128 is supported; Hv must be a multiple of Hqk (value heads
  *     h = j*G .. j*G+G-1 share q/k head j, G = Hv/Hqk).
- *   - The kernels neither normalise q/k nor compute the gates: g is the log-decay
- *     (alpha = exp(g)) and beta the write strength, both per value head.  There is no
- *     scale argument: o = S q literally.
+ *   - gdn_decode / gdn_prefill take the log-decay g (alpha = exp(g)) and the write strength
+ *     beta, both per value head, use q and k as given, and apply no scale: o = S q literally.
+ *     The *_gated entry points compute g and beta from the raw gate inputs inside the kernels;
+ *     the *_fused entry points additionally L2-normalise q and k and scale q (see there).
  */
 #ifndef GDN_H_
 #define GDN_H_
@@ -226,7 +227,17 @@ int gdn_prefill_recurrent(const void* q, const void* k, const void* v, const flo
  * loads the library holds those bytes until the process exits.  Problems whose workspace
  * (gdn_prefill_workspace_bytes) exceeds that size are refused with GDN_ERR_WORKSPACE; nothing
  * is launched in that case.  The call itself performs no cudaMalloc/cudaFree and calls no
- * allocating library routine.
+ * allocating library routine.  The kernels see the scratch 1024-byte aligned, like a caller's
+ * workspace.
+ *
+ * Same values, not the same speed: this entry point always runs the chunked kernels with one
+ * chain per (sequence, value head).  It never cuts long sequences into runs that advance at
+ * the same time (that needs scratch in proportion to the token count) and never hands short
+ * sequences to the token-serial kernel, so few long sequences and very short ones run slower
+ * here than through gdn_prefill.
+ *
+ * Device status: pass workspace = NULL to gdn_last_device_status to read (and clear) the
+ * status word of this scratch on the current device.
  *
  * The first call on each device looks up the array's device address (with that device
  * current) and remembers it; make that first call outside any stream capture.
@@ -285,6 +296,8 @@ int gdn_prefill_apply(const float* S_in, const void* qt, void* out, const int32_
  * Reads (and clears) the device-side status word that the prefill kernels set when a
  * bounded wait on an asynchronous copy or tensor-core completion ran out.  HOST
  * pointer out; synchronises `stream`.  *device_status == 0 means no kernel gave up.
+ * workspace = NULL reads the fixed scratch of gdn_prefill_static on the current device
+ * (GDN_ERR_NULL if gdn_prefill_static has not run on it yet).
  */
 int gdn_last_device_status(void* workspace, int* device_status, void* stream);
 

@@ -4,6 +4,7 @@
 #include <stdlib.h>
 
 #include "gdn_common.cuh"
+#include "gdn_validate.h"
 
 namespace gdn {
 cudaError_t decode_dispatch(const void* q, const void* k, const void* v, const float* g, const float* beta,
@@ -27,6 +28,7 @@ cudaError_t prefill_apply_dispatch(const float* S_in, const void* qt, void* out,
                                    cudaStream_t st);
 cudaError_t launch_state_scan(const float* S0, const float* P, const float* H, int steps, float* S_out, int num_seqs,
                               int Hv, cudaStream_t st);
+void* static_scratch_if_ready();
 cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v, const float* g,
                                      const float* beta, const float* A_log, const float* dt_bias,
                                      const int32_t* cu_seqlens, const float* initial_state,
@@ -34,37 +36,12 @@ cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v
                                      int max_seqlen, int Hqk, int Hv, void* workspace, size_t workspace_bytes,
                                      bool allow_split, QkFront fr, cudaStream_t st);
 
-// 1 = sm_100 family, 0 = other, -1 = unknown yet.  Indexed by device ordinal.
-static int g_device_ok[64] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1,
-                              -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1,
-                              -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1,
-                              -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};
-
-static bool device_supported() {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return false;
-    if (dev < 0 || dev >= 64) return false;
-    if (g_device_ok[dev] < 0) {
-        int major = 0;
-        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
-        g_device_ok[dev] = (major == 10) ? 1 : 0;
-    }
-    return g_device_ok[dev] == 1;
-}
-
 // Maps a CUDA runtime error to a status; with GDN_DEBUG set in the environment the runtime's
 // message goes to stderr (the only case in which the library prints).
 static int cuda_status(cudaError_t e, const char* where) {
     if (e == cudaSuccess) return GDN_OK;
     if (getenv("GDN_DEBUG")) fprintf(stderr, "libgdn: %s: %s\n", where, cudaGetErrorString(e));
     return GDN_ERR_CUDA;
-}
-
-static int check_heads(int Hqk, int Hv, int dk, int dv) {
-    if (Hqk <= 0 || Hv <= 0 || dk <= 0 || dv <= 0) return GDN_ERR_SHAPE;
-    if (Hv % Hqk != 0) return GDN_ERR_SHAPE;
-    if (dk != kD || dv != kD) return GDN_ERR_UNSUPPORTED;
-    return GDN_OK;
 }
 
 static int decode_impl(const void* q, const void* k, const void* v, const float* g, const float* beta,
@@ -83,28 +60,6 @@ static int decode_impl(const void* q, const void* k, const void* v, const float*
     if (!device_supported()) return GDN_ERR_UNSUPPORTED;
     return cuda_status(decode_dispatch(q, k, v, g, beta, gated ? A_log : nullptr, gated ? dt_bias : nullptr, state_in,
                                        state_out, out, B, Hqk, Hv, variant, fr, (cudaStream_t)stream), "gdn_decode");
-}
-
-static int check_prefill(const void* q, const void* k, const void* v, const float* g, const float* beta,
-                         const int32_t* cu_seqlens, const float* initial_state, void* out, float* final_state,
-                         int total_tokens, int num_seqs, int max_seqlen, int Hqk, int Hv, int dk, int dv,
-                         bool* nothing_to_do) {
-    *nothing_to_do = false;
-    if (total_tokens < 0 || num_seqs < 0 || max_seqlen < 0) return GDN_ERR_SHAPE;
-    if (int rc = check_heads(Hqk, Hv, dk, dv)) return rc;
-    if (max_seqlen > total_tokens) return GDN_ERR_SHAPE;
-    if (total_tokens > 0 && (num_seqs == 0 || max_seqlen == 0)) return GDN_ERR_SHAPE;
-    if ((long long)max_seqlen * num_seqs < total_tokens) return GDN_ERR_SHAPE;
-    if (num_seqs == 0) { *nothing_to_do = true; return GDN_OK; }
-    if (!cu_seqlens) return GDN_ERR_NULL;
-    if (total_tokens > 0 && (!q || !k || !v || !g || !beta || !out)) return GDN_ERR_NULL;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) ||
-        !aligned16(out) || !aligned16(initial_state) || !aligned16(final_state) ||
-        (reinterpret_cast<uintptr_t>(cu_seqlens) & 3u))
-        return GDN_ERR_ALIGN;
-    if ((long long)num_seqs * Hv * 16 > 0x7fffffffLL) return GDN_ERR_SHAPE;
-    if (!device_supported()) return GDN_ERR_UNSUPPORTED;
-    return GDN_OK;
 }
 
 // Short-sequence dispatch of gdn_prefill.  When no sequence is longer than one chunk the chunked
@@ -365,7 +320,10 @@ int gdn_prefill_apply(const float* S_in, const void* qt, void* out, const int32_
 }
 
 int gdn_last_device_status(void* workspace, int* device_status, void* stream) {
-    if (!workspace || !device_status) return GDN_ERR_NULL;
+    if (!device_status) return GDN_ERR_NULL;
+    // NULL = the fixed scratch of gdn_prefill_static on the current device (its address is private)
+    if (!workspace) workspace = static_scratch_if_ready();
+    if (!workspace) return GDN_ERR_NULL;
     int val = 0;
     if (cudaMemcpyAsync(&val, workspace, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
         return GDN_ERR_CUDA;

@@ -22,8 +22,10 @@
 //   warp  1     issues every TMA / bulk copy, one chunk ahead of the MMAs
 //   warps 4-7   chain: drain Delta^T -> bf16 operands; drain S -> bf16 operand + decayed fp32 back
 //   warps 8-11  output: drain Oa/Ob -> bf16 out
-//   (warps 2, 3 idle: a role that touches tensor memory needs warp % 4 = its lane quarter)
-// Measured with clock stamps (GDN_CHAIN_PROFILE): a chunk step is ~3150 clocks and stays there when the
+//   warp  2     ragged last chunk only: clears the rows of the V and K tiles that lie beyond the
+//               sequence (the 64-row TMA box also fetched the first tokens of the next sequence)
+//   (warp 3 idle: a role that touches tensor memory needs warp % 4 = its lane quarter)
+// Measured with clock stamps: a chunk step is ~3150 clocks and stays there when the
 // off-chain products are moved around; the drain of Delta^T takes ~590 clocks when no other MMA is issued or
 // executing at the time and 100-300 more when the eight S Q^T MMAs are (in a microbenchmark queued MMAs do
 // not delay another warp's tcgen05.ld / st at all, so this is contention inside the kernel, part of it the
@@ -43,7 +45,7 @@ namespace gdn {
 using namespace sm100;
 
 constexpr int kChainThreads = 384;
-constexpr int kIssuerWarp = 0, kProducerWarp = 1, kChainWarp0 = 4, kOutputWarp0 = 8;  // warps 2, 3 idle
+constexpr int kIssuerWarp = 0, kProducerWarp = 1, kCleanWarp = 2, kChainWarp0 = 4, kOutputWarp0 = 8;  // warp 3 idle
 
 // One arrival per warp: 128 threads arriving on the same mbarrier are serialised by the
 // shared-memory unit (~500 clk before the waiter sees the phase complete); the lanes are ordered
@@ -77,7 +79,7 @@ constexpr uint32_t TM_DTH = 416;    // bf16 (e o Delta)^T hi          32
 constexpr uint32_t TM_DTL = 448;    // bf16 (e o Delta)^T lo          32
 constexpr uint32_t TM_COLS = 512;
 
-enum { B_FULL_A0 = 0, B_FULL_A1, B_FULL_B0, B_FULL_B1, B_FREE0, B_FREE1, B_DELTA, B_STATE, B_O, B_DW, B_SHI, B_STM, B_OFREE, B_DL, B_COUNT };
+enum { B_FULL_A0 = 0, B_FULL_A1, B_FULL_B0, B_FULL_B1, B_FREE0, B_FREE1, B_DELTA, B_STATE, B_O, B_DW, B_SHI, B_STM, B_OFREE, B_DL, B_CLEAN_A, B_CLEAN_B, B_COUNT };
 
 __global__ void __launch_bounds__(kChainThreads, 1)
 gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -87,9 +89,6 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     // CTAs are handed out longest sequence first; within a sequence: run 0, then (zero, identity) per run.
     // Partial mode (part.H set, segs = 1): every sequence is one run that is walked from the zero state
     // and from the identity, results to the caller's H, P and qt.
-#ifdef GDN_CHAIN_PROFILE
-    const uint32_t t_entry = (uint32_t)clock64();
-#endif
     const bool partial = part.H != nullptr;
     const int per_seq = partial ? 2 : 2 * segs - 1;
     const int h = blockIdx.x % Hv, unit = blockIdx.x / Hv;
@@ -132,6 +131,11 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     // chunks of one sequence are consecutive: chunk ci starts at t0_first + 64 ci
     const int t0_first = chunk_info[c_begin].y;
     const int t_end = chunk_info[c_end - 1].y + chunk_info[c_end - 1].z;
+    // Only the last chunk of a run can be ragged.  Its 64-row TMA boxes reach past the sequence into
+    // the next one; those rows meet exact zeros in every product, which is not enough when they hold
+    // NaN or Inf, so they are cleared in shared memory before the tensor cores see them.
+    const int tail_len = t_end - (t0_first + (nchunks - 1) * kChunk);
+    const bool ragged = tail_len < kChunk;
     // where this CTA's state comes from and where its results go
     const size_t state_off = ((size_t)n * Hv + h) * kD * kD;
     const float* init_ptr = (!partial && seg == 0 && initial_state) ? initial_state + state_off : nullptr;
@@ -175,21 +179,6 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     auto scal_ptr = [&](int c) {
         return reinterpret_cast<const float*>(ws + L.off_scal + ((size_t)c * Hv + h) * kScalBytes);
     };
-#ifdef GDN_CHAIN_PROFILE
-#ifndef GDN_CHAIN_PROFILE_CTA
-#define GDN_CHAIN_PROFILE_CTA 0  // the CTA that records
-#endif
-    // SM-clock stamps of one CTA into the unused tail of each chunk's scalar block (4-byte slots from byte 576)
-// GDN_CHAIN_PROFILE is a bit mask of the stamp slots to record (every stamp costs its warp ~150 clocks)
-#define GDN_STAMP(c, slot) do { if ((((unsigned long long)(GDN_CHAIN_PROFILE) >> (slot)) & 1ull) && blockIdx.x == GDN_CHAIN_PROFILE_CTA) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)(c) * Hv + h) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
-#else
-#define GDN_STAMP(c, slot) do { } while (0)
-#endif
-    if (tid == 0) GDN_STAMP(c_begin, 40);  // set-up done (tables read, barriers, tensor memory)
-#ifdef GDN_CHAIN_PROFILE
-    if (tid == 0 && blockIdx.x == GDN_CHAIN_PROFILE_CTA)
-        reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)c_begin * Hv + h) * kScalBytes + 576)[43] = t_entry;
-#endif
 
     if (warp == kIssuerWarp) {
         // =========================================================== issuer: MMA
@@ -201,6 +190,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             const uint32_t tmem_base_u = __shfl_sync(0xffffffffu, tmem_base, 0);
             const int nchunks_u = __shfl_sync(0xffffffffu, nchunks, 0);
             const bool ident_u = __shfl_sync(0xffffffffu, (int)ident, 0) != 0;  // v = 0: no V^T T'^T term
+            const bool ragged_u = __shfl_sync(0xffffffffu, (int)ragged, 0) != 0;
             constexpr uint32_t ID_G1 = umma_idesc_bf16(128, 64, true, false, false);    // V^T (MN-major A) x T'^T
             constexpr uint32_t ID_G2A = umma_idesc_bf16(128, 64, false, false, true);   // -(S) x W^T
             constexpr uint32_t ID_N64 = umma_idesc_bf16(128, 64, false, false, false);  // S x Q^T ; Delta^T x P^T
@@ -236,16 +226,15 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 const int st = ci & 1, par = ci & 1, ph2 = (ci >> 1) & 1;
                 const uint64_t so = st * kStageStep;
                 const bool last = (ci + 1 == nchunks_u);
-                if (lane == 0) GDN_STAMP(c, 0);
                 if (!g1_issued) {
                     GDN_WAIT(B_FULL_A0 + st, ph2);
+                    if (last && ragged_u) GDN_WAIT(B_CLEAN_A, 0);
                     tc_fence_after_sync();
                     if (!ident_u) issue_G1(st);
                 }
                 g1_issued = false;
                 // ---- on the chain: Delta^T -= S W^T   (A = bf16 S in tensor memory)
                 GDN_WAIT(B_SHI, par);
-                if (lane == 0) GDN_STAMP(c, 2);
                 tc_fence_after_sync();
                 {
                     const uint64_t w0 = dW0 + so, w1 = dW1 + so;
@@ -257,7 +246,6 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     for (int ks = 0; ks < 4; ++ks) umma_bf16_ts_warp(td, ta + 32 + ks * 8, w1 + ks * 2, ID_G2A, 1);
                 }
                 umma_commit_warp(bars + B_DELTA);
-                if (lane == 0) GDN_STAMP(c, 4);
                 // ---- off the chain: Oa^T = S Q^T (executes while the chain warps drain Delta^T)
                 if (ci >= 1) GDN_WAIT_READY(B_OFREE, par ^ 1);
                 {
@@ -268,13 +256,11 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) umma_bf16_ts_warp(td, ta + 32 + ks * 8, q1 + ks * 2, ID_N64, 1);
                 }
-                if (lane == 0) GDN_STAMP(c, 5);
                 // ---- on the chain: S += (e o Delta)^T K  (hi + lo; A in tensor memory, B = K MN-major)
                 GDN_WAIT_READY(B_FULL_B0 + st, ph2);
+                if (last && ragged_u) GDN_WAIT_READY(B_CLEAN_B, 0);
                 GDN_WAIT_READY(B_STM, par);
-                if (lane == 0) GDN_STAMP(c, 7);
                 GDN_WAIT(B_DW, par);
-                if (lane == 0) GDN_STAMP(c, 8);
                 tc_fence_after_sync();
                 {
                     const uint64_t k0 = dK + so;
@@ -285,7 +271,6 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     for (int ks = 0; ks < 4; ++ks) umma_bf16_ts_warp(td, tmem_base_u + TM_DTL + ks * 8, k0 + ks * 128, ID_G3B, 1);
                 }
                 umma_commit_warp(bars + B_STATE);
-                if (lane == 0) GDN_STAMP(c, 9);
                 // ---- off the chain: Ob^T = Delta^T P^T, and the next chunk's V^T T'^T if it has landed
                 GDN_WAIT(B_DL, par);
                 tc_fence_after_sync();
@@ -297,12 +282,12 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 umma_commit_warp(bars + B_O);
                 if (!last) {
                     GDN_WAIT_READY(B_FULL_A0 + (st ^ 1), ((ci + 1) >> 1) & 1);  // requested a whole chunk ago
+                    if (ci + 2 == nchunks_u && ragged_u) GDN_WAIT_READY(B_CLEAN_A, 0);
                     tc_fence_after_sync();
                     if (!ident_u) issue_G1(st ^ 1);
                     g1_issued = true;
                 }
                 umma_commit_warp(bars + B_FREE0 + st);  // every MMA that reads this stage has been issued
-                if (lane == 0) GDN_STAMP(c, 10);
             }
 #undef GDN_WAIT
 #undef GDN_WAIT_READY
@@ -358,6 +343,32 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
         }
         __syncwarp();
+    } else if (warp == kCleanWarp) {
+        // =========================================================== ragged last chunk: rows >= tail_len
+        // Rows are tokens, 128 bytes each in both halves of a tile (the swizzle permutes inside a row),
+        // so the rows beyond the sequence are one contiguous range per half tile.
+        if (ragged) {
+            const int lc = nchunks - 1;
+            uint8_t* sp = smem + (lc & 1) * kStageBytes;
+            const uint32_t ph = (uint32_t)((lc >> 1) & 1);
+            const uint32_t from = (uint32_t)tail_len * 128u;
+            auto clear_rows = [&](uint8_t* tile) {
+#pragma unroll 1
+                for (int half = 0; half < 2; ++half)
+                    for (uint32_t o = from + lane * 16u; o < 8192u; o += 512u)
+                        *reinterpret_cast<uint4*>(tile + half * 8192 + o) = make_uint4(0u, 0u, 0u, 0u);
+                fence_proxy_async_smem();  // generic-proxy stores before the tensor cores' reads
+                __syncwarp();
+            };
+            if (mbar_wait_all(bars + B_FULL_A0 + (lc & 1), ph, abort_flag)) {
+                clear_rows(sp + ST_V);
+                if (lane == 0) mbar_arrive(bars + B_CLEAN_A);
+                if (mbar_wait_all(bars + B_FULL_B0 + (lc & 1), ph, abort_flag)) {
+                    clear_rows(sp + ST_K);
+                    if (lane == 0) mbar_arrive(bars + B_CLEAN_B);
+                }
+            }
+        }
     } else if (warp >= kChainWarp0 && warp < kChainWarp0 + 4) {
         // =========================================================== chain warps
         const int v = tid - kChainWarp0 * 32;
@@ -403,7 +414,6 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tc_fence_before_sync();
             warp_arrive(bars + B_SHI);
             warp_arrive(bars + B_STM);
-            if (tid == kChainWarp0 * 32) GDN_STAMP(c_begin, 42);  // initial state in tensor memory
         }
         for (int ci = 0; ci < nchunks; ++ci) {
             const int c = c_begin + ci;
@@ -418,11 +428,8 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 for (int j = 0; j < 16; ++j) ev4[j] = __ldg(e4 + j);
                 if (!last) asm volatile("prefetch.global.L2 [%0];" ::"l"(scal_ptr(c + 1) + (lane & 3) * 32));
             }
-            if (tid == kChainWarp0 * 32) GDN_STAMP(c, 16);
             if (!mbar_wait_all(bars + B_DELTA, par, abort_flag)) break;
             tc_fence_after_sync();
-            if (tid == kChainWarp0 * 32) GDN_STAMP(c, 17);
-            if (lane == 0) GDN_STAMP(c, 36 + (warp & 3));
             // Delta^T row v -> bf16 A operands in tensor memory.  First (e o Delta) as hi + lo, which
             // the state update on the chain is waiting for; the plain bf16 Delta that only the output
             // product needs follows after that hand-off.  Two halves of 32 tokens keep the live
@@ -432,7 +439,6 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 uint32_t r[32], hd[16], ld[16];
                 tmem_ld32(lane_addr + TM_DELTA + half * 32, r);
                 tmem_ld_wait();
-                if (tid == kChainWarp0 * 32 && half == 0) GDN_STAMP(c, 28);
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     const float4 ea = ev4[half * 8 + (j >> 1)];
@@ -445,8 +451,6 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tmem_st_wait();
             tc_fence_before_sync();
             warp_arrive(bars + B_DW);
-            if (tid == kChainWarp0 * 32) GDN_STAMP(c, 18);
-            if (lane == 0) GDN_STAMP(c, 32 + (warp & 3));
             {   // off the chain: bf16 Delta^T for Ob^T = Delta^T P^T (the accumulator is intact until
                 // the next chunk's V^T T'^T, which the issuer starts only after this hand-off)
                 uint32_t r[32], xd[32];
@@ -465,7 +469,6 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
             if (!mbar_wait_all(bars + B_STATE, par, abort_flag)) break;
             tc_fence_after_sync();
-            if (tid == kChainWarp0 * 32) GDN_STAMP(c, 19);
             if (last) {
                 if (fin_ptr) {
                     // run 0 of a split sequence also leaves its final state as the bf16 operand tiles
@@ -509,7 +512,6 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 tmem_st_wait();
                 tc_fence_before_sync();
                 warp_arrive(bars + B_SHI);
-                if (tid == kChainWarp0 * 32) GDN_STAMP(c, 20);
                 // ... then the fp32 state decayed by the next chunk's Gamma_L, in place (gates the next G3B)
 #pragma unroll
                 for (int b = 0; b < 2; ++b) {
@@ -528,7 +530,6 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 tmem_st_wait();
                 tc_fence_before_sync();
                 warp_arrive(bars + B_STM);
-                if (tid == kChainWarp0 * 32) GDN_STAMP(c, 21);
             }
         }
     } else if (warp >= kOutputWarp0) {
@@ -542,10 +543,11 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             auto last_chunk = [&](int i) { return i + 1 == nchunks; };
             const float4* g4 = reinterpret_cast<const float4*>(scal_ptr(c));  // Gamma_i of this chunk
             if (!last_chunk(ci)) asm volatile("prefetch.global.L2 [%0];" ::"l"(scal_ptr(c + 1) + (lane & 1) * 32));
-            if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 24);
-            if (!mbar_wait_all(bars + B_O, par, abort_flag)) break;
+            // A warp whose wait ran out does not leave on its own: the four output warps meet at a named
+            // barrier below, and a warp that had left would strand the others there.  It carries on with
+            // meaningless registers to that barrier, where the four decide together.
+            const bool ok = mbar_wait_all(bars + B_O, par, abort_flag);
             tc_fence_after_sync();
-            if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 25);
             // drain both accumulators into registers and hand the columns back at once: the next
             // chunk's S Q^T is waiting for them
             uint32_t a0[32], a1[32], b0[32], b1[32];
@@ -555,8 +557,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tmem_ld32(lane_addr + TM_OB + 32, b1);
             tmem_ld_wait();
             tc_fence_before_sync();
-            warp_arrive(bars + B_OFREE);
-            if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 26);
+            if (ok) warp_arrive(bars + B_OFREE);
             // o_i = Gamma_i Oa^T[v][i] + Ob^T[v][i], packed two tokens per register
             uint32_t op[32];
 #pragma unroll
@@ -573,20 +574,18 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
             // Through a shared-memory tile so that the global stores are 16 bytes per lane and whole
             // 256-byte rows per half warp (64 two-byte stores per thread kept these warps busier than
-            // the chain itself).  The named barrier covers the four output warps only; every one of
-            // them reaches it in every iteration.
-            if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 44);
+            // the chain itself).  The named barriers cover the four output warps only.  The first one
+            // (the previous chunk's tile has been read) also ANDs the outcome of the wait above over all
+            // 128 threads, so either all four warps go on to the second barrier or all four leave.
             {
                 uint16_t* ost = reinterpret_cast<uint16_t*>(smem + OFF_OST);
-                asm volatile("bar.sync 1, 128;" ::: "memory");  // the previous chunk's tile has been read
+                if (!bar_and(1, 128, ok)) break;
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     ost[(2 * j) * kD + v] = (uint16_t)(op[j] & 0xffffu);
                     ost[(2 * j + 1) * kD + v] = (uint16_t)(op[j] >> 16);
                 }
-                if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 45);
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 46);
                 const int c16 = v & 15, r0 = v >> 4;
                 uint16_t* obase = out_ptr + ((size_t)t0 * Hv + h) * kD + c16 * 8;
                 const size_t ostride = (size_t)Hv * kD;
@@ -598,17 +597,11 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                             *reinterpret_cast<const uint4*>(ost + row * kD + c16 * 8);
                 }
             }
-            if (tid == kOutputWarp0 * 32) GDN_STAMP(c, 27);
         }
     }
 
-    if (tid == 0) GDN_STAMP(c_begin, 41);  // this thread's role is finished
     // ---- unwind: on failure give copies in flight a moment to land, then release tensor memory
-    if (*abort_flag) {
-        const long long t_start = clock64();
-        while (clock64() - t_start < 400000) { }
-        if (tid == 0) atomicExch(reinterpret_cast<int*>(ws), kStatusTimeout);
-    }
+    unwind_after_abort(abort_flag, reinterpret_cast<int*>(ws), kStatusTimeout);
     tc_fence_before_sync();
     __syncthreads();
     if (warp == kIssuerWarp) {

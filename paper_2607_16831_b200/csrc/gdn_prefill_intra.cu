@@ -181,14 +181,6 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int G = Hv / Hqk;
     const int npairs = (G + 1) / 2;
     const int hq = blockIdx.y / npairs, p = blockIdx.y % npairs;
-#ifdef GDN_INTRA_PROFILE
-    // SM-clock stamps of thread 0 into the unused tail of this CTA's first scalar block (4-byte slots from byte 576)
-#define GDN_ISTAMP_T(thread, slot) do { if (threadIdx.x == (thread)) reinterpret_cast<uint32_t*>(ws + L.off_scal + ((size_t)c * Hv + hq * G + 2 * p) * kScalBytes + 576)[slot] = (uint32_t)clock64(); } while (0)
-#else
-#define GDN_ISTAMP_T(thread, slot) do { } while (0)
-#endif
-#define GDN_ISTAMP(slot) GDN_ISTAMP_T(0, slot)
-    GDN_ISTAMP(0);
     const int hh = tid >> 6, i = tid & 63;  // role in the gate / solve / W phases: head of the pair, row
     const int nh = min(2, G - 2 * p);
     const int h = hq * G + 2 * p + hh;      // this thread's value head in those phases
@@ -276,6 +268,18 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     if (warp == 0) {
         ok = mbar_wait_all(bar_load, 0, abort_flag);
         if (ok) {
+            if (len < kChunk) {
+                // Ragged chunk: the 64-row TMA boxes also brought the first tokens of the next sequence.
+                // Their products only ever meet exact zeros (beta = 0, masked decay), which does not stop a
+                // NaN or Inf, so rows >= len of the four tiles are cleared before anything reads them
+                // (128 bytes per row in each tile; the swizzle permutes inside a row).
+#pragma unroll 1
+                for (int tile = 0; tile < 4; ++tile)
+                    for (uint32_t o = (uint32_t)len * 128u + lane * 16u; o < 8192u; o += 512u)
+                        *reinterpret_cast<uint4*>(smem + tile * 8192 + o) = make_uint4(0u, 0u, 0u, 0u);
+                fence_proxy_async_smem();  // generic-proxy stores before the tensor cores' reads
+                __syncwarp();
+            }
             tc_fence_after_sync();
             constexpr uint32_t ID1 = umma_idesc_bf16(128, 64, false, false, false);
             const uint64_t dA0 = umma_desc(sb + IQ_LO, 16, 1024), dA1 = umma_desc(sb + IQ_HI, 16, 1024);
@@ -320,7 +324,6 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     }
     if (warp == 0 && ok) ok = mbar_wait_all(bar_mma1, 0, abort_flag);  // only this warp polls; the others park at the barrier
     ok = __syncthreads_and(ok);
-    GDN_ISTAMP(1);
     if (ok) {
         tc_fence_after_sync();
         // per-token scalars of this thread's (head, row)
@@ -342,9 +345,6 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             const int jb_own = row >> 4;
 #pragma unroll 1
             for (int q4 = 0; q4 < 4; ++q4) {
-                GDN_ISTAMP_T(0, 14 + q4);    // P side (warp 0)
-                GDN_ISTAMP_T(64, 20 + q4);   // A side (warp 2)
-                GDN_ISTAMP_T(96, 26 + q4);   // A side (warp 3)
                 uint32_t r[16];
                 tmem_ld16(lane_addr + ITM_D1 + q4 * 16, r);
                 tmem_ld_wait();
@@ -459,14 +459,10 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
             }
         }
-        GDN_ISTAMP_T(0, 18);
-        GDN_ISTAMP_T(64, 24);
-        GDN_ISTAMP_T(96, 30);
         fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncthreads();  // B tiles and diagonal blocks complete; the accumulator of MMA1 is dead from here on
         tc_fence_after_sync();
-        GDN_ISTAMP(2);
         if constexpr (FRONT) {
             // the tables of the emission below, rescaled in place (phase A is done with them; the solve's
             // barriers come before their next use): beta_j / rk_j and Gamma_j rk_j
@@ -514,7 +510,6 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
             }
             }
-            GDN_ISTAMP(3 + 2 * (3 - jb));
             if (jb > 0) {
                 // this block becomes a K step of the A operand (bf16 hi + lo) for the remaining steps
                 uint32_t zh[8], zl[8];
@@ -544,7 +539,6 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 ok = __syncthreads_and(ok);
                 if (!ok) break;
                 tc_fence_after_sync();
-                GDN_ISTAMP(4 + 2 * (3 - jb));
             }
         }
         // The images that go to the workspace (T' hi, T' lo, W) are row-major with 128-byte rows and a thread
@@ -586,7 +580,6 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             tc_fence_before_sync();
         }
         __syncthreads();
-        GDN_ISTAMP(11);
         const bool storer = ok && i == 0 && head_ok;  // threads 0 and 64: one per head
         if (storer) {
             bulk_store(wsA, stHi, 8192);
@@ -605,7 +598,6 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         }
         if (storer) bulk_store_wait_read();  // the staging of T' hi is written again below
         ok = __syncthreads_and(ok);
-        GDN_ISTAMP(12);
         if (ok) {
             // ---- T' lo (the bf16 remainder, split again from the values kept in registers) -> staging over
             //      the T'' operand, which MMA2 has finished reading
@@ -639,11 +631,9 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 *reinterpret_cast<uint4*>(stW + (b >> 1) * 8192 + swz(i, (b & 1) * 4 + cc)) = o;
             }
         }
-        GDN_ISTAMP(32);
         fence_proxy_async_smem();
     }
     __syncthreads();
-    GDN_ISTAMP(33);
     if (ok && i == 0 && head_ok) {
         uint8_t* wsA = ws + L.off_A + ((size_t)c * Hv + h) * kABytes;
         bulk_store(wsA + 8192, smem + IT2 + (uint32_t)hh * 8192u, 8192);  // T' lo
@@ -652,7 +642,6 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         bulk_store_wait_read();  // shared memory must outlive the copy's reads
     }
 
-    GDN_ISTAMP(13);
     if (*abort_flag && tid == 0) atomicExch(reinterpret_cast<int*>(ws), kStatusTimeout);
     tc_fence_before_sync();
     __syncthreads();

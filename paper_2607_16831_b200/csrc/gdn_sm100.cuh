@@ -58,28 +58,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
                                           long long limit_cycles = 2000000000LL) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long start = clock64();
-#ifndef GDN_WAIT_MODE
-#define GDN_WAIT_MODE 1
-#endif
-    for (uint32_t i = 1;; ++i) {
-#if GDN_WAIT_MODE == 0
-        if (mbar_try_wait(bar, parity)) return true;             // plain polling
-        if ((i & 63u) == 0u) {
-            if (*abort) return false;
-            if (clock64() - start > limit_cycles) break;
-        }
-#elif GDN_WAIT_MODE == 1
-        if (mbar_try_wait(bar, parity, 20000u)) return true;     // sleeps up to 20 us per poll
+    for (;;) {
+        if (mbar_try_wait(bar, parity, 20000u)) return true;  // sleeps up to 20 us per poll
         if (*abort) return false;
         if (clock64() - start > limit_cycles) break;
-#else
-        if (mbar_try_wait(bar, parity)) return true;             // polling with a short back-off
-        __nanosleep(40);
-        if ((i & 15u) == 0u) {
-            if (*abort) return false;
-            if (clock64() - start > limit_cycles) break;
-        }
-#endif
     }
     *abort = 1;
     return false;
@@ -117,6 +99,32 @@ __device__ __forceinline__ bool mbar_wait_all_probe(uint64_t* bar, uint32_t pari
                                                     long long limit_cycles = 2000000000LL) {
     if (__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) return true;
     return mbar_wait_all(bar, parity, abort, limit_cycles);
+}
+
+// Named barrier `id` over `nthreads` threads that also ANDs a predicate over them: every participant
+// gets the same answer, so a decision taken on it (leave a loop or stay) is taken by all of them.
+__device__ __forceinline__ bool bar_and(uint32_t id, uint32_t nthreads, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %3, 0;\n\t"
+        "bar.red.and.pred p, %1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"(id), "r"(nthreads), "r"(pred ? 1u : 0u)
+        : "memory");
+    return r != 0;
+}
+
+// Common tail of a kernel whose roles leave their loops when a bounded wait ran out: on failure the
+// copies that may still be in flight towards this CTA's shared memory get a bounded moment to land
+// and one thread records the time-out in the device status word.  Every thread of the CTA calls it.
+__device__ __forceinline__ void unwind_after_abort(volatile int* abort, int* status_word, int code) {
+    if (*abort) {
+        const long long t_start = clock64();
+        while (clock64() - t_start < 400000) { }
+        if (threadIdx.x == 0 && status_word) atomicExch(status_word, code);
+    }
 }
 
 // ---------------------------------------------------------------- fences

@@ -111,3 +111,88 @@ def test_workspace_size_grows_with_tokens(gdn):
     e = gdn.gdn_prefill_workspace_bytes(8192, 1, 16, 32)
     # few long sequences get extra room for the sequence-parallel scan, so b may exceed c
     assert 0 < a < b < e and a < c < d
+
+
+class _FakeTensor:
+    """Stands in for a CUDA tensor on a box without a GPU: the binding's checks only look at
+    attributes, and every case below is rejected before a pointer is taken."""
+
+    def __init__(self, shape, dtype, strides=None, device="cuda:0", cuda=True):
+        import torch
+
+        self.shape = tuple(shape)
+        self.dtype = dtype
+        self.is_cuda = cuda
+        self.device = torch.device(device)
+        self._contig = strides is None
+        self._strides = strides
+
+    def dim(self):
+        return len(self.shape)
+
+    def is_contiguous(self):
+        return self._contig
+
+    def stride(self):
+        return self._strides or ()
+
+    def data_ptr(self):
+        raise AssertionError("a rejected tensor's pointer must never be taken")
+
+
+def test_binding_rejects_tensors_the_c_abi_would_misread(gdn, monkeypatch):
+    import torch
+
+    monkeypatch.setattr(gdn, "_chk_current", lambda dev: None)
+    bf, f32, i32 = torch.bfloat16, torch.float32, torch.int32
+    B, Hqk, Hv = 2, 2, 4
+    F = _FakeTensor
+
+    def decode_args(**over):
+        a = dict(q=F((B, Hqk, 128), bf), k=F((B, Hqk, 128), bf), v=F((B, Hv, 128), bf), g=F((B, Hv), f32),
+                 beta=F((B, Hv), f32), state_in=F((B, Hv, 128, 128), f32), state_out=F((B, Hv, 128, 128), f32),
+                 out=F((B, Hv, 128), bf))
+        a.update(over)
+        return [a[n] for n in ("q", "k", "v", "g", "beta", "state_in", "state_out", "out")]
+
+    bad = [
+        dict(q=F((B, Hqk, 128), bf, strides=(512, 256, 1))),              # a strided slice such as q[:, ::2]
+        dict(state_in=F((B, Hv, 128, 128), f32, strides=(65536, 16384, 1, 128))),  # a transposed state
+        dict(k=F((B, Hqk, 128), torch.float16)),                          # fp16 is not bf16
+        dict(g=F((B, Hv), torch.float64)),
+        dict(v=F((B, Hv, 128), bf, cuda=False, device="cpu")),
+        dict(out=F((B, Hv, 64), bf)),                                     # wrong head size
+        dict(state_out=F((B + 1, Hv, 128, 128), f32)),                    # batch disagrees
+        dict(beta=F((B, Hv), f32, device="cuda:1")),                      # another device
+        dict(q=None),
+    ]
+    for over in bad:
+        with pytest.raises(ValueError):
+            gdn.gdn_decode(*decode_args(**over))
+
+    T, N = 100, 2
+
+    def prefill_args(**over):
+        a = dict(q=F((T, Hqk, 128), bf), k=F((T, Hqk, 128), bf), v=F((T, Hv, 128), bf), g=F((T, Hv), f32),
+                 beta=F((T, Hv), f32), cu=F((N + 1,), i32), init=F((N, Hv, 128, 128), f32), out=F((T, Hv, 128), bf),
+                 fin=F((N, Hv, 128, 128), f32))
+        a.update(over)
+        return [a[n] for n in ("q", "k", "v", "g", "beta", "cu", "init", "out", "fin")]
+
+    ws = F((1 << 20,), torch.uint8)
+    bad = [
+        dict(cu=F((N + 1,), torch.int64)),                                # int64 offsets
+        dict(init=F((N + 1, Hv, 128, 128), f32)),                         # N disagrees with cu_seqlens
+        dict(fin=F((N, Hv, 128, 128), f32, strides=(1, 1, 1, 1))),
+        dict(out=F((T - 1, Hv, 128), bf)),
+        dict(v=F((T, Hv, 128), bf, strides=(1024, 256, 2))),
+    ]
+    for over in bad:
+        with pytest.raises(ValueError):
+            gdn.gdn_prefill(*prefill_args(**over), 60, ws)
+        with pytest.raises(ValueError):
+            gdn.gdn_prefill_static(*prefill_args(**over), 60)
+    with pytest.raises(ValueError):
+        gdn.gdn_prefill(*prefill_args(), 60, F((1 << 20,), torch.float32))  # the workspace is bytes
+    with pytest.raises(ValueError):
+        gdn.gdn_prefill_gated(*prefill_args()[:5], F((Hv + 1,), f32), F((Hv,), f32), *prefill_args()[5:], 60, ws)
