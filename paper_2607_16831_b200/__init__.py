@@ -149,8 +149,9 @@ def _chk_tokens(q, k, v, g, beta, lead, names=("g", "beta")):
 
 
 def _chk_raw_gates(A_log, dt_bias, Hv, dev, required: bool):
-    _chk("A_log", A_log, "f32", (Hv,), optional=not required, device=dev)
-    _chk("dt_bias", dt_bias, "f32", (Hv,), optional=not required, device=dev)
+    # a missing gate parameter is the library's to report (GDN_ERR_NULL); what is present is checked here
+    _chk("A_log", A_log, "f32", (Hv,), optional=True, device=dev)
+    _chk("dt_bias", dt_bias, "f32", (Hv,), optional=True, device=dev)
 
 
 def _chk_prefill(q, k, v, g, beta, cu_seqlens, initial_state, out, final_state, workspace, names=("g", "beta")):

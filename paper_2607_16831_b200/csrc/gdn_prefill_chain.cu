@@ -22,9 +22,9 @@
 //   warp  1     issues every TMA / bulk copy, one chunk ahead of the MMAs
 //   warps 4-7   chain: drain Delta^T -> bf16 operands; drain S -> bf16 operand + decayed fp32 back
 //   warps 8-11  output: drain Oa/Ob -> bf16 out
-//   warp  2     ragged last chunk only: clears the rows of the V and K tiles that lie beyond the
-//               sequence (the 64-row TMA box also fetched the first tokens of the next sequence)
-//   (warp 3 idle: a role that touches tensor memory needs warp % 4 = its lane quarter)
+//               (and, when the last chunk is ragged, clears the rows of its V and K tiles that lie
+//               beyond the sequence: the 64-row TMA box also fetched the first tokens of the next one)
+//   (warps 2, 3 idle: a role that touches tensor memory needs warp % 4 = its lane quarter)
 // Measured with clock stamps: a chunk step is ~3150 clocks and stays there when the
 // off-chain products are moved around; the drain of Delta^T takes ~590 clocks when no other MMA is issued or
 // executing at the time and 100-300 more when the eight S Q^T MMAs are (in a microbenchmark queued MMAs do
@@ -45,7 +45,7 @@ namespace gdn {
 using namespace sm100;
 
 constexpr int kChainThreads = 384;
-constexpr int kIssuerWarp = 0, kProducerWarp = 1, kCleanWarp = 2, kChainWarp0 = 4, kOutputWarp0 = 8;  // warp 3 idle
+constexpr int kIssuerWarp = 0, kProducerWarp = 1, kChainWarp0 = 4, kOutputWarp0 = 8;  // warps 2, 3 idle
 
 // One arrival per warp: 128 threads arriving on the same mbarrier are serialised by the
 // shared-memory unit (~500 clk before the waiter sees the phase complete); the lanes are ordered
@@ -334,41 +334,44 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 tma_prefetch_3d(&map_k, 64, hq, t0);
             };
             // chunk ci goes to stage ci & 1 as soon as the MMAs of chunk ci - 2 have drained it
+            bool all_requested = true;
             for (int ci = 0; ci < nchunks; ++ci) {
                 if (ci >= 2 &&
-                    !mbar_wait_all(bars + B_FREE0 + (ci & 1), (uint32_t)(((ci >> 1) - 1) & 1), abort_flag))
+                    !mbar_wait_all(bars + B_FREE0 + (ci & 1), (uint32_t)(((ci >> 1) - 1) & 1), abort_flag)) {
+                    all_requested = false;
                     break;
+                }
                 load_all(c_begin + ci, ci & 1);
                 if (ci >= 1 && ci + 1 < nchunks) prefetch_all(c_begin + ci + 1);
             }
-        }
-        __syncwarp();
-    } else if (warp == kCleanWarp) {
-        // =========================================================== ragged last chunk: rows >= tail_len
-        // Rows are tokens, 128 bytes each in both halves of a tile (the swizzle permutes inside a row),
-        // so the rows beyond the sequence are one contiguous range per half tile.
-        if (ragged) {
-            const int lc = nchunks - 1;
-            uint8_t* sp = smem + (lc & 1) * kStageBytes;
-            const uint32_t ph = (uint32_t)((lc >> 1) & 1);
-            const uint32_t from = (uint32_t)tail_len * 128u;
-            auto clear_rows = [&](uint8_t* tile) {
+            // Ragged last chunk: rows >= tail_len of its V and K tiles belong to the next sequence.  Rows are
+            // tokens, 128 bytes each in both halves of a tile (the swizzle permutes inside a row), so they
+            // are one contiguous range per half tile.  This warp armed the stage's barriers for this very
+            // phase a moment ago, so the parity it waits on cannot be mistaken for an earlier use of the stage.
+            if (ragged && all_requested) {
+                const int lc = nchunks - 1;
+                uint8_t* sp = smem + (lc & 1) * kStageBytes;
+                const uint32_t ph = (uint32_t)((lc >> 1) & 1);
+                const uint32_t from = (uint32_t)tail_len * 128u;
+                auto clear_rows = [&](uint8_t* tile) {
 #pragma unroll 1
-                for (int half = 0; half < 2; ++half)
-                    for (uint32_t o = from + lane * 16u; o < 8192u; o += 512u)
-                        *reinterpret_cast<uint4*>(tile + half * 8192 + o) = make_uint4(0u, 0u, 0u, 0u);
-                fence_proxy_async_smem();  // generic-proxy stores before the tensor cores' reads
-                __syncwarp();
-            };
-            if (mbar_wait_all(bars + B_FULL_A0 + (lc & 1), ph, abort_flag)) {
-                clear_rows(sp + ST_V);
-                if (lane == 0) mbar_arrive(bars + B_CLEAN_A);
-                if (mbar_wait_all(bars + B_FULL_B0 + (lc & 1), ph, abort_flag)) {
-                    clear_rows(sp + ST_K);
-                    if (lane == 0) mbar_arrive(bars + B_CLEAN_B);
+                    for (int half = 0; half < 2; ++half)
+                        for (uint32_t o = from + lane * 16u; o < 8192u; o += 512u)
+                            *reinterpret_cast<uint4*>(tile + half * 8192 + o) = make_uint4(0u, 0u, 0u, 0u);
+                    fence_proxy_async_smem();  // generic-proxy stores before the tensor cores' reads
+                    __syncwarp();
+                };
+                if (mbar_wait_all(bars + B_FULL_A0 + (lc & 1), ph, abort_flag)) {
+                    clear_rows(sp + ST_V);
+                    if (lane == 0) mbar_arrive(bars + B_CLEAN_A);
+                    if (mbar_wait_all(bars + B_FULL_B0 + (lc & 1), ph, abort_flag)) {
+                        clear_rows(sp + ST_K);
+                        if (lane == 0) mbar_arrive(bars + B_CLEAN_B);
+                    }
                 }
             }
         }
+        __syncwarp();
     } else if (warp >= kChainWarp0 && warp < kChainWarp0 + 4) {
         // =========================================================== chain warps
         const int v = tid - kChainWarp0 * 32;
@@ -602,8 +605,6 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
     // ---- unwind: on failure give copies in flight a moment to land, then release tensor memory
     unwind_after_abort(abort_flag, reinterpret_cast<int*>(ws), kStatusTimeout);
-    tc_fence_before_sync();
-    __syncthreads();
     if (warp == kIssuerWarp) {
         __syncwarp();
         tmem_dealloc(tmem_base, TM_COLS);

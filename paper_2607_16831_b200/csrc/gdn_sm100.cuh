@@ -116,15 +116,20 @@ __device__ __forceinline__ bool bar_and(uint32_t id, uint32_t nthreads, bool pre
     return r != 0;
 }
 
-// Common tail of a kernel whose roles leave their loops when a bounded wait ran out: on failure the
-// copies that may still be in flight towards this CTA's shared memory get a bounded moment to land
-// and one thread records the time-out in the device status word.  Every thread of the CTA calls it.
+// Common tail of a kernel whose roles leave their loops when a bounded wait ran out.  Every thread of
+// the CTA calls it once its role is finished.  Threads that know of the failure first give the copies
+// that may still be in flight towards this CTA's shared memory a bounded moment to land; then the CTA
+// meets at a barrier (a role that finished early cannot have seen a flag that was raised later, so the
+// flag is only final here) and one thread records the time-out in the device status word.  Tensor
+// memory may be released after the call.
 __device__ __forceinline__ void unwind_after_abort(volatile int* abort, int* status_word, int code) {
     if (*abort) {
         const long long t_start = clock64();
         while (clock64() - t_start < 400000) { }
-        if (threadIdx.x == 0 && status_word) atomicExch(status_word, code);
     }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort && status_word) atomicExch(status_word, code);
 }
 
 // ---------------------------------------------------------------- fences

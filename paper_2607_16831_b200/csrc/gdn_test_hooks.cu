@@ -41,8 +41,6 @@ __global__ void __launch_bounds__(128) gdn_test_bounded_wait_kernel(int* status_
     }
     // ---- the unwind every prefill kernel ends with
     unwind_after_abort(abort_flag, status_word, kStatusTimeout);
-    tc_fence_before_sync();
-    __syncthreads();
     if (warp == 0) {
         __syncwarp();
         tmem_dealloc(tmem_base, 32);
