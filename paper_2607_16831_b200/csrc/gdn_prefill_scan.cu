@@ -190,6 +190,10 @@ gdn_prefill_fixup_kernel(const __grid_constant__ CUtensorMap map_out, const __gr
                          uint16_t* __restrict__ out, uint8_t* __restrict__ ws, WsLayout L, int Hv, int segs,
                          const int* __restrict__ cu, const uint8_t* __restrict__ img_base) {
     const int tid = threadIdx.x, warp = tid >> 5, h = blockIdx.y;
+    // A kernel queued behind this one with programmatic stream serialization (the combine that only
+    // forms the final state, which reads nothing this kernel writes) may start filling SMs as soon as
+    // every CTA of this grid is resident, instead of after the last one has drained.
+    pdl_launch_dependents();
     int t_begin, t_end;
     const uint8_t* img;
     if (cu) {
@@ -303,14 +307,23 @@ gdn_prefill_fixup_kernel(const __grid_constant__ CUtensorMap map_out, const __gr
 // Launch shape of the combine kernel: 16-row CTAs (eight per sequence and head), or 8-row CTAs when even
 // twice as many still leave SMs idle; two P buffers (a whole SM per CTA) when there are several steps and the
 // grid is small enough for it.
-static void launch_combine(const ScanArgs& A, int num_seqs, int Hv, bool several_steps, cudaStream_t st) {
+// `beside_previous`: the kernel before it in the stream neither writes what the combine reads nor reads what
+// it writes, so the combine is queued with programmatic stream serialization and never waits for that grid.
+static void launch_combine(const ScanArgs& A, int num_seqs, int Hv, bool several_steps, cudaStream_t st,
+                           bool beside_previous = false) {
     const long long units = (long long)num_seqs * Hv;
     if (units * 16 <= kAssumedSMs) {
         const int nbuf = several_steps ? 2 : 1;
-        gdn_prefill_combine_kernel<2><<<dim3((unsigned)units, 16), 128, combine_smem(nbuf), st>>>(A, Hv, nbuf);
+        if (beside_previous)
+            launch_pdl(gdn_prefill_combine_kernel<2>, dim3((unsigned)units, 16), dim3(128), combine_smem(nbuf), st, A, Hv, nbuf);
+        else
+            gdn_prefill_combine_kernel<2><<<dim3((unsigned)units, 16), 128, combine_smem(nbuf), st>>>(A, Hv, nbuf);
     } else {
         const int nbuf = (several_steps && units * 8 <= kAssumedSMs) ? 2 : 1;
-        gdn_prefill_combine_kernel<4><<<dim3((unsigned)units, 8), 128, combine_smem(nbuf), st>>>(A, Hv, nbuf);
+        if (beside_previous)
+            launch_pdl(gdn_prefill_combine_kernel<4>, dim3((unsigned)units, 8), dim3(128), combine_smem(nbuf), st, A, Hv, nbuf);
+        else
+            gdn_prefill_combine_kernel<4><<<dim3((unsigned)units, 8), 128, combine_smem(nbuf), st>>>(A, Hv, nbuf);
     }
 }
 
@@ -357,7 +370,7 @@ cudaError_t launch_prefill_scan(const CUtensorMap& mout, const CUtensorMap& mqt,
     const dim3 fgrid((unsigned)((seg_chunks * kChunk + kFixTokens - 1) / kFixTokens), (unsigned)Hv,
                      (unsigned)(num_seqs * (segs - 1)));
     gdn_prefill_fixup_kernel<<<fgrid, 128, kFixSmem, st>>>(mout, mqt, (uint16_t*)out, ws, L, Hv, segs, nullptr, nullptr);
-    if (segs == 2 && final_state) launch_combine(A, num_seqs, Hv, false, st);
+    if (segs == 2 && final_state) launch_combine(A, num_seqs, Hv, false, st, true);  // runs beside the fix-up
     return cudaGetLastError();
 }
 
