@@ -79,11 +79,12 @@ constexpr uint32_t TM_DTH = 416;    // bf16 (e o Delta)^T hi          32
 constexpr uint32_t TM_DTL = 448;    // bf16 (e o Delta)^T lo          32
 constexpr uint32_t TM_COLS = 512;
 
-enum { B_FULL_A0 = 0, B_FULL_A1, B_FULL_B0, B_FULL_B1, B_FREE0, B_FREE1, B_DELTA, B_STATE, B_O, B_DW, B_SHI, B_STM, B_OFREE, B_DL, B_CLEAN_A, B_CLEAN_B, B_COUNT };
+enum { B_FULL_A0 = 0, B_FULL_A1, B_FULL_B0, B_FULL_B1, B_FREE0, B_FREE1, B_DELTA, B_STATE, B_O, B_DW, B_SHI, B_STM, B_OFREE, B_DL, B_CLEAN_A, B_CLEAN_B, B_INIT, B_INIT_DONE, B_COUNT };
 
 __global__ void __launch_bounds__(kChainThreads, 1)
 gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                         const __grid_constant__ CUtensorMap map_v, const float* initial_state,
+                         const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_s,
+                         const float* initial_state,
                          uint16_t* __restrict__ out, float* final_state, uint8_t* __restrict__ ws, WsLayout L,
                          int Hqk, int Hv, int segs, ChainPartial part) {
     // CTAs are handed out longest sequence first; within a sequence: run 0, then (zero, identity) per run.
@@ -92,7 +93,10 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const bool partial = part.H != nullptr;
     const int per_seq = partial ? 2 : 2 * segs - 1;
     const int h = blockIdx.x % Hv, unit = blockIdx.x / Hv;
-    const int n = reinterpret_cast<const int*>(ws + L.off_seq_order)[unit / per_seq];
+    // one record per sequence (sequence, its first chunk, its first token, its length): everything this CTA
+    // needs to find its work comes from this single load
+    const int4 rec = reinterpret_cast<const int4*>(ws + L.off_seq_order)[unit / per_seq];
+    const int n = rec.x;
     const int seg = partial ? 0 : (unit % per_seq + 1) >> 1;
     const bool ident = partial ? (unit % per_seq) == 1
                                : (seg > 0 && ((unit % per_seq) & 1) == 0);  // identity start, v = 0
@@ -105,11 +109,12 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 8 * B_COUNT);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_BAR + 8 * B_COUNT + 8);
 
-    const int* chunk_off = reinterpret_cast<const int*>(ws + L.off_chunk_off);
-    const int4* chunk_info = reinterpret_cast<const int4*>(ws + L.off_chunk_info);
+    // chunk slots of the sequence, clamped like the chunk table itself (a malformed cu_seqlens cannot
+    // send the CTA outside the workspace)
+    const int seq_chunks = max(0, min((rec.w + kChunk - 1) / kChunk, L.nc_max - rec.y));
     int seg_first, nchunks;
-    segment_range(chunk_off[n + 1] - chunk_off[n], segs, seg, seg_first, nchunks);
-    const int c_begin = chunk_off[n] + seg_first, c_end = c_begin + nchunks;
+    segment_range(seq_chunks, segs, seg, seg_first, nchunks);
+    const int c_begin = rec.y + seg_first;
 
     if (nchunks <= 0) {  // empty sequence: the state passes through; empty run: nothing to do
         if (partial && tid < kD) {  // H = 0, P = I
@@ -128,9 +133,9 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         }
         return;
     }
-    // chunks of one sequence are consecutive: chunk ci starts at t0_first + 64 ci
-    const int t0_first = chunk_info[c_begin].y;
-    const int t_end = chunk_info[c_end - 1].y + chunk_info[c_end - 1].z;
+    // chunks of one sequence are consecutive: chunk ci of this run starts at t0_first + 64 ci
+    const int t0_first = rec.z + seg_first * kChunk;
+    const int t_end = min(rec.z + rec.w, t0_first + nchunks * kChunk);
     // Only the last chunk of a run can be ragged.  Its 64-row TMA boxes reach past the sequence into
     // the next one; those rows meet exact zeros in every product, which is not enough when they hold
     // NaN or Inf, so they are cleared in shared memory before the tensor cores see them.
@@ -147,21 +152,11 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             ws + seg_block_offset(L, n, seg == 0 ? 1 : seg, h, Hv, seg == 0 ? kSegSin : (ident ? kSegP : kSegH)));
     uint16_t* out_ptr = ident ? (partial ? part.qt : reinterpret_cast<uint16_t*>(ws + L.off_qt)) : out;
 
-    // The chain warps will read their rows of the initial state (thread v: row v, four 128-byte lines) once
-    // the barriers and the tensor memory are set up; the lines are asked into L2 now, so that those
-    // loads do not pay the DRAM latency after the set-up.
-    if (warp >= kChainWarp0 && warp < kChainWarp0 + 4) {
-        if (init_ptr) {
-            const char* row = reinterpret_cast<const char*>(init_ptr + (size_t)(tid - kChainWarp0 * 32) * kD);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) prefetch_l2(row + 128 * j);
-        }
-        if ((tid & 31) == 0)
-            prefetch_l2(ws + L.off_scal + ((size_t)c_begin * Hv + h) * kScalBytes + 512);
-    }
+    if (warp >= kChainWarp0 && warp < kChainWarp0 + 4 && (tid & 31) == 0)
+        prefetch_l2(ws + L.off_scal + ((size_t)c_begin * Hv + h) * kScalBytes + 512);
     if (tid == 0) {
         for (int i = 0; i < B_COUNT; ++i) {
-            const bool many = (i == B_DW || i == B_SHI || i == B_STM || i == B_OFREE || i == B_DL);
+            const bool many = (i == B_DW || i == B_SHI || i == B_STM || i == B_OFREE || i == B_DL || i == B_INIT_DONE);
             mbar_init(bars + i, many ? 4u : 1u);  // one arrival per warp of the arriving role
         }
         *abort_flag = 0;
@@ -333,11 +328,24 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 tma_prefetch_3d(&map_k, 0, hq, t0);
                 tma_prefetch_3d(&map_k, 64, hq, t0);
             };
+            // The initial state (64 KB, fp32) comes in as four [128 rows][32 floats] boxes with the 128-byte
+            // swizzle, into the second stage's buffers, which nothing else needs before the second chunk:
+            // one bulk transfer that overlaps the rest of the set-up, where 128 lanes each reading their
+            // own 512-byte row used to take several microseconds.  The chain warps lift it into tensor memory.
+            if (init_ptr && elect_one()) {
+                mbar_expect_tx(bars + B_INIT, 4u * 16384u);
+                const int row0 = (int)(state_off / kD);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    tma_load_2d(smem + kStageBytes + j * 16384, &map_s, bars + B_INIT, 32 * j, row0);
+            }
+            __syncwarp();
             // chunk ci goes to stage ci & 1 as soon as the MMAs of chunk ci - 2 have drained it
             bool all_requested = true;
             for (int ci = 0; ci < nchunks; ++ci) {
-                if (ci >= 2 &&
-                    !mbar_wait_all(bars + B_FREE0 + (ci & 1), (uint32_t)(((ci >> 1) - 1) & 1), abort_flag)) {
+                if ((ci >= 2 &&
+                     !mbar_wait_all(bars + B_FREE0 + (ci & 1), (uint32_t)(((ci >> 1) - 1) & 1), abort_flag)) ||
+                    (ci == 1 && init_ptr && !mbar_wait_all(bars + B_INIT_DONE, 0, abort_flag))) {
                     all_requested = false;
                     break;
                 }
@@ -380,15 +388,21 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         // initial state: bf16 operand copy and Gamma_L(first chunk) * S, both into tensor memory
         {
             const float gl0 = __ldg(scal_ptr(c_begin) + 128);
+            bool have_init = init_ptr != nullptr;
+            if (have_init) have_init = mbar_wait_all(bars + B_INIT, 0, abort_flag);  // (on failure: zeros, and the loop below leaves)
+            // row v of box jb sits at v * 128 in that box, its 16-byte piece c at (c ^ (v & 7)) * 16: the
+            // eight lanes of a quarter warp hit eight different 16-byte bank groups
+            const uint8_t* srow = smem + kStageBytes + (uint32_t)v * 128u;
 #pragma unroll 1
             for (int b = 0; b < 2; ++b) {
                 uint32_t r0[32], r1[32], pk[32];
 #pragma unroll
                 for (int j = 0; j < 32; j += 4) {
                     float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
-                    if (init_ptr) {
-                        x = *reinterpret_cast<const float4*>(init_ptr + sbase + b * 64 + j);
-                        y = *reinterpret_cast<const float4*>(init_ptr + sbase + b * 64 + 32 + j);
+                    if (have_init) {
+                        const uint32_t piece = (uint32_t)(((j >> 2) ^ (v & 7)) << 4);
+                        x = *reinterpret_cast<const float4*>(srow + (2 * b) * 16384 + piece);
+                        y = *reinterpret_cast<const float4*>(srow + (2 * b + 1) * 16384 + piece);
                     } else if (ident) {
                         const int d0 = v - (b * 64 + j), d1 = d0 - 32;  // the one of row v sits in column v
                         x = make_float4(d0 == 0 ? 1.f : 0.f, d0 == 1 ? 1.f : 0.f, d0 == 2 ? 1.f : 0.f, d0 == 3 ? 1.f : 0.f);
@@ -413,6 +427,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 tmem_st32(lane_addr + TM_S + b * 64, r0);
                 tmem_st32(lane_addr + TM_S + b * 64 + 32, r1);
             }
+            if (init_ptr) warp_arrive(bars + B_INIT_DONE);  // the second stage's buffers may be filled now
             tmem_st_wait();
             tc_fence_before_sync();
             warp_arrive(bars + B_SHI);
@@ -612,7 +627,7 @@ gdn_prefill_chain_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 }
 
 cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                                 const float* initial_state, void* out, float* final_state, uint8_t* ws,
+                                 const CUtensorMap& ms, const float* initial_state, void* out, float* final_state, uint8_t* ws,
                                  const WsLayout& L, int num_seqs, int Hqk, int Hv, int segs, const ChainPartial& part,
                                  cudaStream_t st) {
     static bool attr_done[64];
@@ -622,7 +637,7 @@ cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, c
         return e;
     const int per_seq = part.H ? 2 : 2 * segs - 1;
     gdn_prefill_chain_kernel<<<(unsigned)((long long)num_seqs * per_seq * Hv), kChainThreads, kChainSmem, st>>>(
-        mq, mk, mv, initial_state, (uint16_t*)out, final_state, ws, L, Hqk, Hv, segs, part);
+        mq, mk, mv, ms, initial_state, (uint16_t*)out, final_state, ws, L, Hqk, Hv, segs, part);
     return cudaGetLastError();
 }
 

@@ -61,6 +61,19 @@ static bool make_map(CUtensorMap* m, const void* base, int T, int H) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 states [rows][128] -> boxes of 128 rows x 32 floats (128 bytes), 128-byte swizzle.
+static bool make_state_map(CUtensorMap* m, const float* base, long long rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)kD * 4};
+    cuuint32_t box[2] = {32, 128};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v, const float* g,
                                      const float* beta, const float* A_log, const float* dt_bias,
                                      const int32_t* cu_seqlens, const float* initial_state,
@@ -82,7 +95,10 @@ cudaError_t prefill_chunked_dispatch(const void* q, const void* k, const void* v
                                  total_tokens, fr, st);
         if (e != cudaSuccess) return e;
         const int segs = choose_segments(L, num_seqs, Hv, max_seqlen);
-        e = launch_prefill_chain(mq, mk, mv, initial_state, out, final_state, ws, L, num_seqs, Hqk, Hv, segs,
+        CUtensorMap ms;
+        memset(&ms, 0, sizeof ms);
+        if (initial_state && !make_state_map(&ms, initial_state, (long long)num_seqs * Hv * kD)) return cudaErrorUnknown;
+        e = launch_prefill_chain(mq, mk, mv, ms, initial_state, out, final_state, ws, L, num_seqs, Hqk, Hv, segs,
                                  ChainPartial{nullptr, nullptr, nullptr}, st);
         if (e != cudaSuccess) return e;
         if (segs > 1) {
@@ -128,7 +144,7 @@ cudaError_t prefill_partial_dispatch(const void* q, const void* k, const void* v
         mk = mq;
         mv = mq;
     }
-    return launch_prefill_chain(mq, mk, mv, nullptr, out0, nullptr, ws, L, num_seqs, Hqk, Hv, 1,
+    return launch_prefill_chain(mq, mk, mv, mq, nullptr, out0, nullptr, ws, L, num_seqs, Hqk, Hv, 1,
                                 ChainPartial{H, P, static_cast<uint16_t*>(qt)}, st);
 }
 

@@ -19,7 +19,7 @@ using namespace sm100;
 // ------------------------------------------------------------------ prep: chunk table
 __global__ void __launch_bounds__(256)
 gdn_prefill_prep_kernel(const int32_t* __restrict__ cu, int num_seqs, int total_tokens, int* hdr,
-                        int* chunk_off, int* seq_order, int4* chunk_info, int nc_max) {
+                        int* chunk_off, int4* seq_order, int4* chunk_info, int nc_max) {
     __shared__ int part[257];
     const int tid = threadIdx.x;
     const int per = (num_seqs + 255) / 256;
@@ -58,14 +58,19 @@ gdn_prefill_prep_kernel(const int32_t* __restrict__ cu, int num_seqs, int total_
     // Longest sequences first: the chain kernel runs one CTA per (sequence, head) and its cost is
     // the chunk count, so handing out the long chains first shortens the tail of the launch.
     // Rank by counting (ties broken by index); O(N^2 / 256) per thread is fine for any sane batch.
+    // The record holds everything a chain CTA needs to know about its sequence, so that it finds its
+    // work with one load instead of a chain of dependent ones.
+    __syncthreads();  // chunk_off of every sequence is written
     for (int n = tid; n < num_seqs; n += 256) {
-        const int ln = max(0, min(cu[n + 1], total_tokens)) - max(0, min(cu[n], total_tokens));
+        const int tn = max(0, min(cu[n], total_tokens));
+        const int ln = max(tn, min(cu[n + 1], total_tokens)) - tn;
         int rank = 0;
         for (int m = 0; m < num_seqs; ++m) {
-            const int lm = max(0, min(cu[m + 1], total_tokens)) - max(0, min(cu[m], total_tokens));
+            const int tm = max(0, min(cu[m], total_tokens));
+            const int lm = max(tm, min(cu[m + 1], total_tokens)) - tm;
             rank += (lm > ln) || (lm == ln && m < n);
         }
-        seq_order[rank] = n;
+        seq_order[rank] = make_int4(n, chunk_off[n], tn, ln);
     }
 }
 
@@ -146,7 +151,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         if (blockIdx.x == 0 && blockIdx.y == 0) {
             int* hdr_w = reinterpret_cast<int*>(ws);
             int* chunk_off = reinterpret_cast<int*>(ws + L.off_chunk_off);
-            int* seq_order = reinterpret_cast<int*>(ws + L.off_seq_order);
+            int4* seq_order = reinterpret_cast<int4*>(ws + L.off_seq_order);
             int4* chunk_info = reinterpret_cast<int4*>(ws + L.off_chunk_info);
             const int total = min(run, L.nc_max);
             if (tid == 0) {
@@ -163,7 +168,7 @@ gdn_prefill_intra_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     rank += (bm - am > b - a) || (bm - am == b - a && m < n);
                 }
                 chunk_off[n] = min(base, L.nc_max);
-                seq_order[rank] = n;  // longest first
+                seq_order[rank] = make_int4(n, min(base, L.nc_max), a, b - a);  // longest first
                 const int nch = (b - a + kChunk - 1) / kChunk;
                 for (int j = 0; j < nch; ++j)
                     if (base + j < L.nc_max)
@@ -655,7 +660,7 @@ cudaError_t launch_prefill_prep(const int32_t* cu_seqlens, int num_seqs, int tot
                                 const WsLayout& L, cudaStream_t st) {
     gdn_prefill_prep_kernel<<<1, 256, 0, st>>>(cu_seqlens, num_seqs, total_tokens, reinterpret_cast<int*>(ws),
                                                reinterpret_cast<int*>(ws + L.off_chunk_off),
-                                               reinterpret_cast<int*>(ws + L.off_seq_order),
+                                               reinterpret_cast<int4*>(ws + L.off_seq_order),
                                                reinterpret_cast<int4*>(ws + L.off_chunk_info), L.nc_max);
     return cudaGetLastError();
 }

@@ -53,8 +53,8 @@ __host__ __device__ inline WsLayout ws_layout(int total_tokens, int num_seqs, in
     size_t o = 1024;                              // header: [0] status, [1] total chunks
     L.off_chunk_off = o;
     o = align_up(o + sizeof(int) * (size_t)(num_seqs + 1), 1024);
-    L.off_seq_order = o;                          // sequences by decreasing chunk count
-    o = align_up(o + sizeof(int) * (size_t)num_seqs, 1024);
+    L.off_seq_order = o;   // sequences by decreasing length: int4 (sequence, its first chunk, its first token, its length)
+    o = align_up(o + sizeof(int4) * (size_t)num_seqs, 1024);
     L.off_chunk_info = o;
     o = align_up(o + sizeof(int4) * (size_t)L.nc_max, 1024);
     L.off_scal = o;
@@ -99,8 +99,10 @@ struct ChainPartial {
 };
 
 // `segs` > 1 splits every sequence into that many runs of chunks (see gdn_prefill_scan.cu).
+// `ms`: tensor map over the initial states as fp32 [num_seqs * Hv * 128 rows][128], boxes of 128 rows x 32
+// floats with the 128-byte swizzle (unused, may be zero-filled, when initial_state is NULL).
 cudaError_t launch_prefill_chain(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                                 const float* initial_state, void* out, float* final_state, uint8_t* ws,
+                                 const CUtensorMap& ms, const float* initial_state, void* out, float* final_state, uint8_t* ws,
                                  const WsLayout& L, int num_seqs, int Hqk, int Hv, int segs, const ChainPartial& part,
                                  cudaStream_t st);
 cudaError_t launch_prefill_scan(const CUtensorMap& mout, const CUtensorMap& mqt, void* out, float* final_state,
