@@ -139,6 +139,12 @@ size_t gdn_prefill_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int 
  * The number of runs follows from num_seqs, Hv and max_seqlen; the environment variable
  * GDN_PREFILL_MAX_SEGMENTS (1..8) lowers it, 1 switches the split off.
  *
+ * Many short sequences (more chains than SMs, at most ~10 chunks per sequence on average) are
+ * walked by persistent thread blocks, one per SM, that keep their barriers and tensor memory from
+ * one chain to the next and fetch the next chain's operands while the current one finishes; what
+ * that saves is per chain, so long chains keep one thread block per chain.
+ * GDN_PREFILL_PERSISTENT=0/1 in the environment forces one form (same results either way).
+ *
  * At the other end, when max_seqlen <= 64 (no sequence longer than one chunk) and a cost model
  * fitted to measurements says the token-serial kernel of gdn_prefill_recurrent is faster (a few
  * short sequences, or many sequences of a handful of tokens), gdn_prefill runs that kernel

@@ -272,3 +272,15 @@ def test_prefill_does_not_depend_on_what_the_workspace_and_outputs_held(lengths,
     for o, f in got[1:]:
         np.testing.assert_array_equal(o, got[0][0])
         np.testing.assert_array_equal(f, got[0][1])
+
+
+@pytest.mark.parametrize("persistent", ["0", "1"])
+@pytest.mark.parametrize("lengths,Hqk,Hv", [([70, 0, 1, 200, 64, 129, 5, 300], 2, 4), ([64] * 40 + [1, 65], 1, 8),
+                                            ([1100, 40, 700], 1, 2)])
+def test_prefill_chain_kernel_forms_agree_with_the_oracle(monkeypatch, persistent, lengths, Hqk, Hv):
+    """The chain kernel has two forms -- one thread block per chain, or persistent thread blocks that walk
+    several chains each (what gdn_prefill picks for many short sequences).  Both are forced here on batches
+    that mix empty, one-token, ragged and multi-chunk sequences (and, in the last case, sequences that are
+    cut into runs), with more chains than the persistent form has thread blocks in the second case."""
+    monkeypatch.setenv("GDN_PREFILL_PERSISTENT", persistent)
+    check(custom(lengths, Hqk, Hv, seed=41, gate_mean=4.0), "prefill, persistent=%s, %d sequences" % (persistent, len(lengths)))
