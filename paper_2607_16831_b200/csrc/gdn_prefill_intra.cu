@@ -55,22 +55,38 @@ gdn_prefill_prep_kernel(const int32_t* __restrict__ cu, int num_seqs, int total_
             if (base + j < nc_max) chunk_info[base + j] = make_int4(n, t0 + j * kChunk, min(kChunk, t1 - t0 - j * kChunk), j);
         base += nch;
     }
-    // Longest sequences first: the chain kernel runs one CTA per (sequence, head) and its cost is
-    // the chunk count, so handing out the long chains first shortens the tail of the launch.
-    // Rank by counting (ties broken by index); O(N^2 / 256) per thread is fine for any sane batch.
-    // The record holds everything a chain CTA needs to know about its sequence, so that it finds its
+    // Longest sequences first: the chain kernel's cost per chain is the chunk count, so handing out the
+    // long chains first shortens the tail of the launch.  Rank by counting (ties broken by index), the
+    // lengths of 256 sequences at a time staged in shared memory: O(N^2 / 256) shared-memory reads per
+    // thread.  The record holds everything a chain needs to know about its sequence, so that it finds its
     // work with one load instead of a chain of dependent ones.
     __syncthreads();  // chunk_off of every sequence is written
-    for (int n = tid; n < num_seqs; n += 256) {
-        const int tn = max(0, min(cu[n], total_tokens));
-        const int ln = max(tn, min(cu[n + 1], total_tokens)) - tn;
-        int rank = 0;
-        for (int m = 0; m < num_seqs; ++m) {
-            const int tm = max(0, min(cu[m], total_tokens));
-            const int lm = max(tm, min(cu[m + 1], total_tokens)) - tm;
-            rank += (lm > ln) || (lm == ln && m < n);
+    __shared__ int len_s[256];
+    for (int n0 = 0; n0 < num_seqs; n0 += 256) {   // (uniform trip count: every thread takes part in the staging)
+        const int n = n0 + tid;
+        int tn = 0, ln = -1;
+        if (n < num_seqs) {
+            tn = max(0, min(cu[n], total_tokens));
+            ln = max(tn, min(cu[n + 1], total_tokens)) - tn;
         }
-        seq_order[rank] = make_int4(n, chunk_off[n], tn, ln);
+        int rank = 0;
+        for (int m0 = 0; m0 < num_seqs; m0 += 256) {
+            __syncthreads();
+            const int m = m0 + tid;
+            int lm = -1;
+            if (m < num_seqs) {
+                const int tm = max(0, min(cu[m], total_tokens));
+                lm = max(tm, min(cu[m + 1], total_tokens)) - tm;
+            }
+            len_s[tid] = lm;
+            __syncthreads();
+            const int cnt = min(256, num_seqs - m0);
+            for (int j = 0; j < cnt; ++j) {
+                const int l = len_s[j];
+                rank += (l > ln) || (l == ln && m0 + j < n);
+            }
+        }
+        if (n < num_seqs) seq_order[rank] = make_int4(n, chunk_off[n], tn, ln);
     }
 }
 

@@ -3,6 +3,7 @@
   python -m paper_2607_16831_b200.profile_target --workload decode --B 64 --calls 3
   python -m paper_2607_16831_b200.profile_target --workload prefill_long --T 1024 --calls 2
   python -m paper_2607_16831_b200.profile_target --workload prefill_varlen --calls 2
+  python -m paper_2607_16831_b200.profile_target --workload prefill_short --calls 2   (256 x 64 tokens, 4/8 heads)
 """
 from __future__ import annotations
 
@@ -17,7 +18,7 @@ sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--workload", default="decode", choices=["decode", "prefill_long", "prefill_varlen", "prefill_tiny"])
+    ap.add_argument("--workload", default="decode", choices=["decode", "prefill_long", "prefill_varlen", "prefill_tiny", "prefill_short"])
     ap.add_argument("--B", type=int, default=64)
     ap.add_argument("--T", type=int, default=4096)
     ap.add_argument("--Hqk", type=int, default=16)
@@ -47,8 +48,15 @@ def main():
             gdn.gdn_decode(d["q"], d["k"], d["v"], d["g"], d["beta"], a, b, out)
             ev[i][1].record()
     else:
-        over = {"T": args.T, "initial": args.initial} if args.workload == "prefill_long" else {}
-        cfg = config(args.workload, Hqk=args.Hqk, Hv=args.Hv, **over)
+        if args.workload == "prefill_short":
+            # many short sequences at the contest's head counts: 256 sequences of 64 tokens, 4 key / 8 value heads
+            from gdn_inputs import make_cu_seqlens, make_state, make_tokens
+            lengths = [64] * 256
+            cfg = dict(tokens=make_tokens(sum(lengths), 4, 8, seed=0), cu_seqlens=make_cu_seqlens(lengths),
+                       initial_state=make_state(len(lengths), 8, seed=0))
+        else:
+            over = {"T": args.T, "initial": args.initial} if args.workload == "prefill_long" else {}
+            cfg = config(args.workload, Hqk=args.Hqk, Hv=args.Hv, **over)
         tok = cfg["tokens"]
         d = harness.to_device(tok)
         cu_np = np.asarray(cfg["cu_seqlens"], dtype=np.int32)
