@@ -526,10 +526,15 @@ def run_gpu(args):
                 auto = bench_prefill("short", peaks, 8, lengths=[ln] * nseq, Hqk=4, Hv=8)["us"]
                 chunked = bench_prefill("short", peaks, 8, lengths=[ln] * nseq, Hqk=4, Hv=8,
                                         env={"GDN_PREFILL_SHORT_FALLBACK": "0"})["us"]
+                per_chain = bench_prefill("short", peaks, 8, lengths=[ln] * nseq, Hqk=4, Hv=8,
+                                          env={"GDN_PREFILL_SHORT_FALLBACK": "0", "GDN_PREFILL_PERSISTENT": "0"})["us"]
                 sweep_short.append({"num_seqs": nseq, "len": ln, "us": auto, "us_chunked_forced": chunked,
+                                    "us_chunked_one_block_per_chain": per_chain,
                                     "tokens_per_s": nseq * ln / (auto * 1e-6)})
             short_sweep_result = {"heads": "4/8", "note": "cold single calls; equal `us` means the chunked path was "
-                                                         "chosen by the dispatch (always so above 64 tokens)",
+                                                         "chosen by the dispatch (always so above 64 tokens); "
+                                                         "`us_chunked_one_block_per_chain` switches the persistent "
+                                                         "chain kernel off (GDN_PREFILL_PERSISTENT=0)",
                                   "points": sweep_short}
             # Where whole 64-token chunks cost the most: sequences just over one chunk, whose second chunk is
             # mostly padding.  Each point is timed against the same number of sequences at the next multiple of
