@@ -124,6 +124,9 @@ size_t gdn_prefill_workspace_bytes(int total_tokens, int num_seqs, int Hqk, int 
  *                 max_seqlen must be >= the longest sequence and <= total_tokens
  *   workspace     >= gdn_prefill_workspace_bytes(...) bytes, 1024-byte aligned
  *
+ * Sequences of a batch do not influence each other, whatever their values: a NaN or Inf in
+ * one sequence's tokens stays in that sequence's outputs and state.
+ *
  * A malformed cu_seqlens can give wrong results but never an out-of-range access:
  * every token index is clamped to [0, total_tokens).  total_tokens = 0 or
  * num_seqs = 0 returns GDN_OK without launching.

@@ -1,11 +1,12 @@
 // Inter-chunk ("chain") kernel of the chunked WY / UT-transform prefill.
 //
-// A chain = one (sequence, value head) whose 64-token chunks are walked in order.  The kernel is
-// persistent: one CTA per SM takes chains from a list sorted by decreasing length (dealt out in a
-// snake so that every CTA gets about the same number of chunk steps) and walks them one after the
-// other, keeping its barriers and its tensor memory; the copy warp runs ahead into the next chain,
-// so that chain's first operands and its initial state are on their way while this chain's last
-// chunk is still being computed and its final state stored.  With
+// A chain = one (sequence, value head) whose 64-token chunks are walked in order.  The kernel has
+// two forms (template parameter): one CTA per chain, or persistent -- one CTA per SM takes chains
+// from a list sorted by decreasing length (dealt out in a snake so that every CTA gets about the
+// same number of chunk steps) and walks them one after the other, keeping its barriers and its
+// tensor memory; the copy warp runs ahead into the next chain, so that chain's first operands and
+// its initial state are on their way while this chain's last chunk is still being computed and its
+// final state stored.  launch_prefill_chain says when which form is used.  With
 // S the fp32 state entering a chunk ([dv][dk], row v = tensor-memory lane v) and the chunk
 // summaries T', W, P and scalars from the intra-chunk kernel:
 //
@@ -24,11 +25,14 @@
 // pre-swizzled images, two stages deep.  The fp32 state stays in tensor memory for the
 // whole sequence.  Warp roles:
 //   warp  0     issues every MMA (one elected lane)
-//   warp  1     issues every TMA / bulk copy, one chunk ahead of the MMAs
-//   warps 4-7   chain: drain Delta^T -> bf16 operands; drain S -> bf16 operand + decayed fp32 back
+//   warp  1     issues every TMA / bulk copy, one chunk ahead of the MMAs (the chain's initial state
+//               included: one swizzled 64 KB transfer into the buffers of the stage its second chunk
+//               will use); when a chain's last chunk is ragged it also clears the rows of that chunk's
+//               V and K tiles that lie beyond the sequence (the 64-row TMA box also fetched the first
+//               tokens of the next one, and zeros in the other operand do not stop a NaN)
+//   warps 4-7   chain: initial state -> tensor memory; drain Delta^T -> bf16 operands; drain S -> bf16
+//               operand + decayed fp32 back; final state -> global memory
 //   warps 8-11  output: drain Oa/Ob -> bf16 out
-//               (and, when the last chunk is ragged, clears the rows of its V and K tiles that lie
-//               beyond the sequence: the 64-row TMA box also fetched the first tokens of the next one)
 //   (warps 2, 3 idle: a role that touches tensor memory needs warp % 4 = its lane quarter)
 // Measured with clock stamps: a chunk step is ~3150 clocks and stays there when the
 // off-chain products are moved around; the drain of Delta^T takes ~590 clocks when no other MMA is issued or

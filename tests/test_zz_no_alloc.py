@@ -90,3 +90,11 @@ def test_static_scratch_prefill_refuses_oversized_problems():
     with pytest.raises(gdn.GdnError) as err:
         gdn.gdn_prefill_static(q, q, v, gb, gb, cu, None, out, None, T)
     assert err.value.status == 4  # GDN_ERR_WORKSPACE
+
+
+def test_static_scratch_status_word_is_readable_only_after_a_static_call():
+    """The scratch's address is private to the library; gdn_last_device_status(None) reads its status word."""
+    import paper_2607_16831_b200 as gdn
+
+    # (after the tests above the scratch of this device has been looked up: the read succeeds and is clean)
+    assert gdn.gdn_last_device_status(None) == 0
