@@ -92,9 +92,10 @@ def test_static_scratch_prefill_refuses_oversized_problems():
     assert err.value.status == 4  # GDN_ERR_WORKSPACE
 
 
-def test_static_scratch_status_word_is_readable_only_after_a_static_call():
-    """The scratch's address is private to the library; gdn_last_device_status(None) reads its status word."""
+def test_static_scratch_status_word_is_readable():
+    """The scratch's address is private to the library; gdn_last_device_status(None) reads its status word
+    (a static call comes first, so the test also stands alone in a fresh process)."""
     import paper_2607_16831_b200 as gdn
 
-    # (after the tests above the scratch of this device has been looked up: the read succeeds and is clean)
+    _run_both([70], 1, 1, 3)
     assert gdn.gdn_last_device_status(None) == 0
